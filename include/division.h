@@ -1,0 +1,162 @@
+/*
+ * division.h -- C ABI of the B200 DIVISION activation compress / decompress library.
+ *
+ * The operation is the per-layer pair of DIVISION ("Memory Efficient Training via Dual
+ * Activation Precision"), Sec. 4.1 "Activation Map Compression" and Sec. 4.2 "Activation Map
+ * Decompression" (Algorithm 1, lines 3-6 and 10-11):
+ *
+ *   compress    H^L = AveragePooling(H), window = stride = B                    (Sec. 4.1)
+ *               H^H = H - UpSampling(H^L), nearest interpolation                (Sec. 4.1)
+ *               V^H = stochastic_round((H^H - delta) / Delta), Q bits           (Eq. 9)
+ *               delta = min H^H,  Delta = (max H^H - delta) / (2^Q - 1)
+ *   decompress  H_hat = UpSampling(H^L) + Delta * V^H + delta                   (Sec. 4.2, Eq. 10)
+ *
+ * for an activation map H of shape N x C x H x W (the paper's Minibatch x Channel x N x N),
+ * contiguous NCHW, fp32 or bf16.
+ *
+ * Conventions fixed by this library where the paper is silent (the same rules are written out in
+ * the CPU checker, which was implemented separately):
+ *   - one (delta, Delta) pair per SAMPLE, kept in fp32;
+ *   - H or W not divisible by B: ceil grid, partial tiles average their in-bounds elements
+ *     (a side shorter than B gives a 1 x 1 map, as the paper's footnote in Sec. 4.1 requires);
+ *   - the residual is taken against the stored (rounded) low-frequency value;
+ *   - rounding up happens with probability frac(t), t = (H^H - delta) * (2^Q - 1)/(max - min);
+ *     the uniform number of element e of sample n is a pure function of (seed, n, e)
+ *     ("DIVRNG-v1": one 64-bit mix per 4 elements, 16-bit uniforms);
+ *   - all arithmetic is IEEE fp32, one rounding per operation, no fused multiply-add, and the
+ *     block sum uses a fixed order (pairwise tree down the rows, then across the columns), so
+ *     the output is a pure function of (descriptor, input bits, seed): independent of grid
+ *     size, SM count and timing;
+ *   - codes of 32/Q consecutive elements (global NCHW flat order) share one little-endian 32-bit
+ *     word, first element in the lowest bits.
+ *
+ * Compressed buffer ("blob"), one caller-owned device allocation:
+ *     [ lfc : N*C*ceil(H/B)*ceil(W/B) values of lfc_dtype | pad to 128 B |
+ *       packed : ceil(N*C*H*W*Q/32) uint32 words          | pad to 128 B |
+ *       stats  : N pairs (delta, Delta) fp32 ]
+ *
+ * Ownership and behaviour common to all entry points:
+ *   - every pointer named *_dev is DEVICE memory owned by the caller, 16-byte aligned;
+ *     descriptors and layouts are HOST memory;
+ *   - the library allocates nothing and keeps no state between calls;
+ *   - div_compress / div_decompress only enqueue work on the given CUDA stream (a cudaStream_t
+ *     passed as void*; NULL is the default stream) and return; errors that can be seen on the
+ *     host are returned at once and nothing is launched;
+ *   - inputs must be finite.  x is never modified; outputs may not alias inputs.
+ */
+#ifndef DIVISION_H_
+#define DIVISION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum div_status {
+    DIV_OK = 0,
+    DIV_ERR_NULL = 1,      /* a required pointer is NULL                                   */
+    DIV_ERR_SHAPE = 2,     /* n, c, h or w < 1, or c*h*w >= 2^32, or n >= 2^31             */
+    DIV_ERR_PARAM = 3,     /* block < 1, qbits not in {1,2,4,8}, unknown dtype or flag     */
+    DIV_ERR_ALIGN = 4,     /* a device pointer is not 16-byte aligned                      */
+    DIV_ERR_CAPACITY = 5,  /* blob or workspace smaller than div_compressed_bytes reports  */
+    DIV_ERR_CUDA = 6,      /* the CUDA runtime reported an error (launch, attribute, ...)  */
+    DIV_ERR_TIMEOUT = 7    /* device side: a bounded wait inside the fused kernel ran out  */
+} div_status;
+
+typedef enum div_dtype { DIV_F32 = 0, DIV_BF16 = 1 } div_dtype;
+
+/* Problem statement: tensor shape, block size B, bit width Q, dtypes (Sec. 4.1). */
+typedef struct div_desc {
+    int64_t n, c, h, w;   /* all >= 1; c*h*w < 2^32; n < 2^31                            */
+    int32_t block;        /* B >= 1 (the paper uses 8; also 4, 12, 16, 18, 64)           */
+    int32_t qbits;        /* Q in {1, 2, 4, 8} (the paper uses 2, 4, 8)                  */
+    int32_t x_dtype;      /* div_dtype of x and of x_hat                                 */
+    int32_t lfc_dtype;    /* div_dtype the low-frequency map is stored in                */
+} div_desc;
+
+/* Byte layout of the blob and of the scratch workspace; all offsets from the blob start. */
+typedef struct div_layout {
+    uint64_t lfc_off, lfc_bytes;
+    uint64_t packed_off, packed_bytes;
+    uint64_t stats_off, stats_bytes;
+    uint64_t total_bytes;        /* blob size to allocate (includes alignment padding)          */
+    uint64_t closed_form_bytes;  /* lfc_bytes + packed_bytes + stats_bytes (what the ratio uses) */
+    uint64_t raw_bytes;          /* n*c*h*w*sizeof(x_dtype)                                      */
+    uint64_t workspace_bytes;    /* scratch div_compress needs (per-sample min/max/arrival slots) */
+} div_layout;
+
+/* How div_compress will run a descriptor (introspection for tests and benchmarks). */
+typedef struct div_plan {
+    int32_t fused;          /* 1: single fused pass over x;  0: two-pass general kernels      */
+    int32_t grid;           /* CTAs of the (first) compress kernel                            */
+    int32_t threads;        /* threads per CTA                                                */
+    int32_t stages;         /* shared-memory ring depth (fused only)                          */
+    int32_t lag;            /* chunks between min/max and quantise of the same chunk (fused)  */
+    int32_t smem_bytes;     /* dynamic shared memory per CTA                                  */
+    int64_t chunk_elems;    /* elements per full chunk (fused only)                           */
+    int64_t chunks_per_sample;
+    int32_t decompress_fast;/* 1: vectorised decompress kernel applies                        */
+    int32_t reserved;
+} div_plan;
+
+/* flags of div_compress_ex */
+#define DIV_FLAG_FORCE_TWO_PASS 1u   /* never take the fused kernel */
+
+/*
+ * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:
+ *   closed form = N*C*ceil(H/B)*ceil(W/B)*sizeof(lfc) + ceil(N*C*H*W*Q/32)*4 + 8*N.
+ * Host only, pure integer arithmetic, never touches a device.
+ * desc, out: host pointers.  Returns DIV_ERR_NULL / DIV_ERR_SHAPE / DIV_ERR_PARAM on bad input.
+ */
+div_status div_compressed_bytes(const div_desc* desc, div_layout* out);
+
+/*
+ * Compress one activation map (Sec. 4.1; Algorithm 1 lines 3-6).
+ *   desc           host; the problem statement
+ *   x_dev          device; N*C*H*W values of x_dtype, contiguous NCHW; read only
+ *   comp_dev       device; receives the blob; at least layout.total_bytes
+ *   comp_capacity  bytes available at comp_dev
+ *   workspace_dev  device scratch of at least layout.workspace_bytes; contents on entry are
+ *                  irrelevant (the call clears it on the stream); after the call its first word
+ *                  holds a device-side status (see div_read_device_status)
+ *   workspace_bytes bytes available at workspace_dev
+ *   seed           seed of the stochastic rounding
+ *   cuda_stream    cudaStream_t as void*
+ * Two calls that overlap on the GPU must not share a workspace.
+ */
+div_status div_compress(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                        void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream);
+
+/* Same as div_compress with DIV_FLAG_* bits (0 = default behaviour). */
+div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                           void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream,
+                           uint32_t flags);
+
+/*
+ * Decompress (Sec. 4.2; Algorithm 1 lines 10-11): x_hat = UpSampling(H^L) + Delta*V^H + delta,
+ * rounded to x_dtype.
+ *   comp_dev    device; a blob written by div_compress with the SAME desc; read only
+ *   comp_bytes  bytes valid at comp_dev (>= layout.total_bytes)
+ *   xhat_dev    device; receives N*C*H*W values of x_dtype, contiguous NCHW
+ */
+div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes,
+                          void* xhat_dev, void* cuda_stream);
+
+/* Which kernels a descriptor maps to on the current device.  desc, out: host. */
+div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
+
+/*
+ * Device-side status of the last div_compress that used this workspace: synchronises the stream,
+ * copies one word back.  *out_status is DIV_OK or DIV_ERR_TIMEOUT.  Host-blocking.
+ */
+div_status div_read_device_status(const void* workspace_dev, void* cuda_stream, int32_t* out_status);
+
+/* Static, NUL-terminated description of a status code. */
+const char* div_status_string(div_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DIVISION_H_ */

@@ -332,8 +332,13 @@ class Compressed:
 
 
 def compress(x: np.ndarray, block: int, qbits: int, seed: int,
-             x_dtype: str = F32, lfc_dtype: str = F32) -> Compressed:
-    """Algorithm 1 lines 3-6 for one activation map H of shape N x C x H x W."""
+             x_dtype: str = F32, lfc_dtype: str = F32, first_sample: int = 0) -> Compressed:
+    """Algorithm 1 lines 3-6 for one activation map H of shape N x C x H x W.
+
+    `first_sample`: x holds samples first_sample, first_sample+1, ... of a larger mini-batch (samples
+    are independent, so a slice of a batch can be checked alone; only the random stream depends on
+    the sample's index in the batch).
+    """
     if qbits not in SUPPORTED_QBITS:
         raise ValueError("Q must divide 32")
     x32 = widen_input(x, x_dtype)
@@ -347,7 +352,7 @@ def compress(x: np.ndarray, block: int, qbits: int, seed: int,
     e = np.arange(chw, dtype=np.uint64)
     for i in range(n):                                                   # line 5, per sample
         delta[i], step[i], scale = sample_stats(r[i], qbits)
-        codes[i] = quantize(r[i], delta[i], scale, divrng_fields(seed, i, e), qbits)
+        codes[i] = quantize(r[i], delta[i], scale, divrng_fields(seed, first_sample + i, e), qbits)
     words = pack_codes(codes.reshape(-1), qbits)
     layout = compressed_layout(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
     return Compressed((n, c, h, w), block, qbits, x_dtype, lfc_dtype, lfc, codes, words, delta, step, layout)

@@ -1,0 +1,182 @@
+"""ctypes binding of libdivision.so: the same entry points as include/division.h, argument marshalling only.
+
+Every step of compress / decompress runs inside the CUDA library.  PyTorch appears here only as the
+owner of device memory and streams.  If the library has not been built the import of the symbols
+fails loudly; nothing falls back to the CPU.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_int32, c_int64, c_size_t, c_uint32, c_uint64, c_void_p
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdivision.so")
+
+DIV_OK = 0
+DIV_ERR_NULL, DIV_ERR_SHAPE, DIV_ERR_PARAM, DIV_ERR_ALIGN, DIV_ERR_CAPACITY, DIV_ERR_CUDA, DIV_ERR_TIMEOUT = range(1, 8)
+DIV_F32, DIV_BF16 = 0, 1
+DIV_FLAG_FORCE_TWO_PASS = 1
+DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
+
+EXPORTED_SYMBOLS = (
+    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_decompress", "div_plan_query",
+    "div_read_device_status", "div_status_string",
+)
+
+
+class DivDesc(ctypes.Structure):
+    _fields_ = [("n", c_int64), ("c", c_int64), ("h", c_int64), ("w", c_int64),
+                ("block", c_int32), ("qbits", c_int32), ("x_dtype", c_int32), ("lfc_dtype", c_int32)]
+
+
+class DivLayout(ctypes.Structure):
+    _fields_ = [(name, c_uint64) for name in (
+        "lfc_off", "lfc_bytes", "packed_off", "packed_bytes", "stats_off", "stats_bytes",
+        "total_bytes", "closed_form_bytes", "raw_bytes", "workspace_bytes")]
+
+
+class DivPlan(ctypes.Structure):
+    _fields_ = [("fused", c_int32), ("grid", c_int32), ("threads", c_int32), ("stages", c_int32),
+                ("lag", c_int32), ("smem_bytes", c_int32), ("chunk_elems", c_int64),
+                ("chunks_per_sample", c_int64), ("decompress_fast", c_int32), ("reserved", c_int32)]
+
+
+class DivisionError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library; raises if it was never built (there is no other implementation to run)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2208_04187_b200.build` "
+                "(or __graft_entry__.build()); this package has no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        L.div_compressed_bytes.argtypes = [ctypes.POINTER(DivDesc), ctypes.POINTER(DivLayout)]
+        L.div_compressed_bytes.restype = c_int32
+        L.div_compress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_void_p, c_size_t, c_void_p, c_size_t,
+                                   c_uint64, c_void_p]
+        L.div_compress.restype = c_int32
+        L.div_compress_ex.argtypes = L.div_compress.argtypes + [c_uint32]
+        L.div_compress_ex.restype = c_int32
+        L.div_decompress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_size_t, c_void_p, c_void_p]
+        L.div_decompress.restype = c_int32
+        L.div_plan_query.argtypes = [ctypes.POINTER(DivDesc), c_uint32, ctypes.POINTER(DivPlan)]
+        L.div_plan_query.restype = c_int32
+        L.div_read_device_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_int32)]
+        L.div_read_device_status.restype = c_int32
+        L.div_status_string.argtypes = [c_int32]
+        L.div_status_string.restype = c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().div_status_string(int(status)).decode()
+
+
+def make_desc(n, c, h, w, block, qbits, x_dtype="f32", lfc_dtype="f32") -> DivDesc:
+    return DivDesc(int(n), int(c), int(h), int(w), int(block), int(qbits),
+                   DTYPE_CODES[x_dtype], DTYPE_CODES[lfc_dtype])
+
+
+def _check(status: int, where: str):
+    if status != DIV_OK:
+        raise DivisionError(status, where)
+
+
+def div_compressed_bytes(desc: DivDesc) -> DivLayout:
+    out = DivLayout()
+    _check(lib().div_compressed_bytes(ctypes.byref(desc), ctypes.byref(out)), "div_compressed_bytes")
+    return out
+
+
+def div_plan_query(desc: DivDesc, flags: int = 0) -> DivPlan:
+    out = DivPlan()
+    _check(lib().div_plan_query(ctypes.byref(desc), int(flags), ctypes.byref(out)), "div_plan_query")
+    return out
+
+
+def div_compress(desc: DivDesc, x_ptr: int, comp_ptr: int, comp_capacity: int, ws_ptr: int, ws_bytes: int,
+                 seed: int, stream: int = 0, flags: int = 0) -> None:
+    """Raw-pointer call (device pointers as integers, stream as a cudaStream_t handle)."""
+    st = lib().div_compress_ex(ctypes.byref(desc), c_void_p(x_ptr), c_void_p(comp_ptr), comp_capacity,
+                               c_void_p(ws_ptr), ws_bytes, c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream),
+                               int(flags))
+    _check(st, "div_compress")
+
+
+def div_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xhat_ptr: int, stream: int = 0) -> None:
+    st = lib().div_decompress(ctypes.byref(desc), c_void_p(comp_ptr), comp_bytes, c_void_p(xhat_ptr),
+                              c_void_p(stream))
+    _check(st, "div_decompress")
+
+
+def div_read_device_status(ws_ptr: int, stream: int = 0) -> int:
+    out = c_int32(0)
+    _check(lib().div_read_device_status(c_void_p(ws_ptr), c_void_p(stream), ctypes.byref(out)),
+           "div_read_device_status")
+    return out.value
+
+
+# ----------------------------------------------------------------------------------------
+# torch conveniences: buffers and pointers only
+# ----------------------------------------------------------------------------------------
+def _torch():
+    import torch
+    return torch
+
+
+def torch_dtype(name: str):
+    torch = _torch()
+    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+
+
+def current_stream_handle() -> int:
+    return int(_torch().cuda.current_stream().cuda_stream)
+
+
+class Codec:
+    """Device buffers for one descriptor (blob, workspace) and the two calls on torch tensors."""
+
+    def __init__(self, n, c, h, w, block, qbits, x_dtype="f32", lfc_dtype="f32", device="cuda"):
+        torch = _torch()
+        self.x_dtype, self.lfc_dtype = x_dtype, lfc_dtype
+        self.desc = make_desc(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
+        self.layout = div_compressed_bytes(self.desc)
+        self.shape = (n, c, h, w)
+        self.device = torch.device(device)
+        self.blob = torch.zeros(int(self.layout.total_bytes), dtype=torch.uint8, device=self.device)
+        self.workspace = torch.zeros(int(self.layout.workspace_bytes), dtype=torch.uint8, device=self.device)
+
+    def plan(self, flags: int = 0) -> DivPlan:
+        return div_plan_query(self.desc, flags)
+
+    def compress(self, x, seed: int = 0, flags: int = 0, blob=None):
+        """x: contiguous CUDA tensor of shape N x C x H x W in the descriptor's dtype."""
+        torch = _torch()
+        blob = self.blob if blob is None else blob
+        if not (x.is_cuda and x.is_contiguous() and tuple(x.shape) == self.shape
+                and x.dtype == torch_dtype(self.x_dtype)):
+            raise ValueError("x must be a contiguous CUDA tensor matching the descriptor")
+        div_compress(self.desc, x.data_ptr(), blob.data_ptr(), blob.numel(), self.workspace.data_ptr(),
+                     self.workspace.numel(), seed, current_stream_handle(), flags)
+        return blob
+
+    def decompress(self, blob=None, out=None):
+        torch = _torch()
+        blob = self.blob if blob is None else blob
+        if out is None:
+            out = torch.empty(self.shape, dtype=torch_dtype(self.x_dtype), device=self.device)
+        div_decompress(self.desc, blob.data_ptr(), blob.numel(), out.data_ptr(), current_stream_handle())
+        return out
+
+    def device_status(self) -> int:
+        return div_read_device_status(self.workspace.data_ptr(), current_stream_handle())

@@ -1,0 +1,276 @@
+// Host side of the C ABI declared in include/division.h: argument checks, byte-layout arithmetic,
+// kernel selection and launches.  Nothing here allocates device memory or keeps state.
+#include "../../include/division.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "common.cuh"
+#include "decompress.cuh"
+#include "fused.cuh"
+#include "twopass.cuh"
+
+namespace {
+
+using namespace divk;
+typedef __nv_bfloat16 bf16;
+
+constexpr uint64_t SECTION_ALIGN = 128;
+
+inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
+
+div_status check_desc(const div_desc* d) {
+    if (!d) return DIV_ERR_NULL;
+    if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return DIV_ERR_SHAPE;
+    if (d->n >= (1ll << 31) || d->c >= (1ll << 32) || d->h >= (1ll << 32) || d->w >= (1ll << 32)) return DIV_ERR_SHAPE;
+    // c*h*w < 2^32 (width of the random-number counter), checked without overflow
+    const unsigned __int128 chw = (unsigned __int128)d->c * (unsigned __int128)d->h * (unsigned __int128)d->w;
+    if (chw >= ((unsigned __int128)1 << 32)) return DIV_ERR_SHAPE;
+    if (d->block < 1) return DIV_ERR_PARAM;
+    if (!(d->qbits == 1 || d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return DIV_ERR_PARAM;
+    if (!(d->x_dtype == DIV_F32 || d->x_dtype == DIV_BF16)) return DIV_ERR_PARAM;
+    if (!(d->lfc_dtype == DIV_F32 || d->lfc_dtype == DIV_BF16)) return DIV_ERR_PARAM;
+    return DIV_OK;
+}
+
+Shape make_shape(const div_desc* d) {
+    Shape s;
+    s.N = (uint32_t)d->n;
+    s.C = (uint32_t)d->c;
+    s.H = (uint32_t)d->h;
+    s.W = (uint32_t)d->w;
+    // a block larger than both sides behaves like a block equal to the larger side
+    const uint32_t big = s.H > s.W ? s.H : s.W;
+    s.B = (uint32_t)d->block > big ? big : (uint32_t)d->block;
+    s.Hb = (s.H + s.B - 1) / s.B;
+    s.Wb = (s.W + s.B - 1) / s.B;
+    s.P2 = 1;
+    while (s.P2 < s.B) s.P2 <<= 1;
+    s.HW = s.H * s.W;
+    s.CHW = s.C * s.HW;
+    s.TPP = s.Hb * s.Wb;
+    s.total = (uint64_t)s.N * s.CHW;
+    s.tiles = (uint64_t)s.N * s.C * s.TPP;
+    return s;
+}
+
+void make_layout(const div_desc* d, const Shape& s, div_layout* out) {
+    out->lfc_off = 0;
+    out->lfc_bytes = s.tiles * dtype_bytes(d->lfc_dtype);
+    out->packed_off = align_up(out->lfc_bytes, SECTION_ALIGN);
+    // ceil(total*Q/32) words; total*Q < 2^31 * 2^32 * 8 fits in 64 bits
+    out->packed_bytes = ((s.total * (uint64_t)d->qbits + 31) / 32) * 4;
+    out->stats_off = align_up(out->packed_off + out->packed_bytes, SECTION_ALIGN);
+    out->stats_bytes = 8ull * s.N;
+    out->total_bytes = out->stats_off + out->stats_bytes;
+    out->closed_form_bytes = out->lfc_bytes + out->packed_bytes + out->stats_bytes;
+    out->raw_bytes = s.total * dtype_bytes(d->x_dtype);
+    out->workspace_bytes = align_up(4ull * (WS_HEADER_WORDS + (uint64_t)WS_SLOT_WORDS * s.N), 256);
+}
+
+FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    f.d = d;
+    uint32_t s = 0;
+    while ((1ull << s) < d) ++s;
+    f.shift = 31 + s;
+    f.mul = (uint32_t)((((1ull << f.shift) - 1) / d) + 1);
+    return f;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------------------------------
+// dispatch helpers: runtime (dtype, dtype, Q) -> template instance
+// ------------------------------------------------------------------------------------------
+template <typename F>
+div_status dispatch_q(int qbits, F&& f) {
+    switch (qbits) {
+        case 1: return f(std::integral_constant<int, 1>());
+        case 2: return f(std::integral_constant<int, 2>());
+        case 4: return f(std::integral_constant<int, 4>());
+        case 8: return f(std::integral_constant<int, 8>());
+    }
+    return DIV_ERR_PARAM;
+}
+template <typename F>
+div_status dispatch_types(int x_dtype, int lfc_dtype, F&& f) {
+    if (x_dtype == DIV_F32) {
+        if (lfc_dtype == DIV_F32) return f((float*)nullptr, (float*)nullptr);
+        return f((float*)nullptr, (bf16*)nullptr);
+    }
+    if (lfc_dtype == DIV_F32) return f((bf16*)nullptr, (float*)nullptr);
+    return f((bf16*)nullptr, (bf16*)nullptr);
+}
+
+inline div_status launch_status() { return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA; }
+
+// ------------------------------------------------------------------------------------------
+// two-pass compress
+// ------------------------------------------------------------------------------------------
+div_status compress_two_pass(const div_desc* d, const Shape& s, const div_layout& lo, const void* x, uint8_t* blob,
+                             uint32_t* ws, uint64_t seed, cudaStream_t st) {
+    const uint64_t nwords = lo.packed_bytes / 4;
+    const uint64_t g1 = (s.tiles + 255) / 256, g2 = (nwords + 255) / 256;
+    if (g1 > 0x7FFFFFFFull || g2 > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
+    return dispatch_types(d->x_dtype, d->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        lfc_stats_kernel<XT, LT><<<(unsigned)g1, 256, 0, st>>>((const XT*)x, (LT*)(blob + lo.lfc_off), ws, s);
+        if (launch_status() != DIV_OK) return DIV_ERR_CUDA;
+        return dispatch_q(d->qbits, [&](auto q) -> div_status {
+            quant_pack_kernel<XT, LT, decltype(q)::value><<<(unsigned)g2, 256, 0, st>>>(
+                (const XT*)x, (const LT*)(blob + lo.lfc_off), ws, (uint32_t*)(blob + lo.packed_off),
+                (float*)(blob + lo.stats_off), s, seed, nwords);
+            return launch_status();
+        });
+    });
+}
+
+// ------------------------------------------------------------------------------------------
+// decompress
+// ------------------------------------------------------------------------------------------
+constexpr int DEC_QPT = 4;
+
+bool decompress_fast_ok(const Shape& s) {
+    return (s.W % 4 == 0) && s.B >= 4 && (s.B & (s.B - 1)) == 0 && s.N <= 65535;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* div_status_string(div_status s) {
+    switch (s) {
+        case DIV_OK: return "ok";
+        case DIV_ERR_NULL: return "null pointer";
+        case DIV_ERR_SHAPE: return "bad shape (need n,c,h,w >= 1, c*h*w < 2^32, n < 2^31)";
+        case DIV_ERR_PARAM: return "bad parameter (block >= 1, qbits in {1,2,4,8}, dtype in {f32,bf16})";
+        case DIV_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case DIV_ERR_CAPACITY: return "buffer too small";
+        case DIV_ERR_CUDA: return "CUDA runtime error";
+        case DIV_ERR_TIMEOUT: return "device-side bounded wait expired";
+    }
+    return "unknown status";
+}
+
+div_status div_compressed_bytes(const div_desc* desc, div_layout* out) {
+    if (!desc || !out) return DIV_ERR_NULL;
+    const div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    make_layout(desc, make_shape(desc), out);
+    return DIV_OK;
+}
+
+div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
+    if (!desc || !out) return DIV_ERR_NULL;
+    const div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    const Shape s = make_shape(desc);
+    *out = div_plan();
+    FusedPlan fp;
+    const bool fused = !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
+    out->fused = fused ? 1 : 0;
+    if (fused) {
+        out->grid = fp.grid;
+        out->threads = fp.threads;
+        out->stages = fp.stages;
+        out->lag = fp.lag;
+        out->smem_bytes = fp.smem_bytes;
+        out->chunk_elems = fp.chunk_elems;
+        out->chunks_per_sample = fp.chunks_per_sample;
+    } else {
+        out->grid = (int32_t)((s.tiles + 255) / 256);
+        out->threads = 256;
+    }
+    out->decompress_fast = decompress_fast_ok(s) ? 1 : 0;
+    return DIV_OK;
+}
+
+div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                           void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream,
+                           uint32_t flags) {
+    if (!desc || !x_dev || !comp_dev || !workspace_dev) return DIV_ERR_NULL;
+    div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    if (!aligned16(x_dev) || !aligned16(comp_dev) || !aligned16(workspace_dev)) return DIV_ERR_ALIGN;
+    const Shape s = make_shape(desc);
+    div_layout lo;
+    make_layout(desc, s, &lo);
+    if (comp_capacity < lo.total_bytes || workspace_bytes < lo.workspace_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
+    uint8_t* blob = (uint8_t*)comp_dev;
+    uint32_t* ws = (uint32_t*)workspace_dev;
+    if (!(flags & DIV_FLAG_FORCE_TWO_PASS)) {
+        FusedPlan fp;
+        if (plan_fused(desc, s, &fp) == DIV_OK) return compress_fused(desc, s, lo, fp, x_dev, blob, ws, seed, stream);
+    }
+    return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
+}
+
+div_status div_compress(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                        void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream) {
+    return div_compress_ex(desc, x_dev, comp_dev, comp_capacity, workspace_dev, workspace_bytes, seed, cuda_stream, 0u);
+}
+
+div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes, void* xhat_dev,
+                          void* cuda_stream) {
+    if (!desc || !comp_dev || !xhat_dev) return DIV_ERR_NULL;
+    div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (!aligned16(comp_dev) || !aligned16(xhat_dev)) return DIV_ERR_ALIGN;
+    const Shape s = make_shape(desc);
+    div_layout lo;
+    make_layout(desc, s, &lo);
+    if (comp_bytes < lo.total_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const uint8_t* blob = (const uint8_t*)comp_dev;
+    const uint64_t nwords = lo.packed_bytes / 4;
+    return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+            constexpr int Q = decltype(q)::value;
+            const LT* lfc = (const LT*)(blob + lo.lfc_off);
+            const uint32_t* packed = (const uint32_t*)(blob + lo.packed_off);
+            const float* stats = (const float*)(blob + lo.stats_off);
+            if (decompress_fast_ok(s)) {
+                DecFast d;
+                d.qps = s.CHW / 4;
+                d.C = s.C;
+                d.TPP = s.TPP;
+                d.Wb = s.Wb;
+                d.log2B = 0;
+                while ((1u << d.log2B) < s.B) ++d.log2B;
+                d.hwq = s.HW / 4;
+                d.wq = s.W / 4;
+                d.by_hwq = make_fastdiv(d.hwq);
+                d.by_wq = make_fastdiv(d.wq);
+                const uint32_t per_block = 256u * DEC_QPT;
+                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+            } else {
+                const uint64_t g = (nwords + 255) / 256;
+                if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
+                decompress_general_kernel<XT, LT, Q><<<(unsigned)g, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, s, nwords);
+            }
+            return launch_status();
+        });
+    });
+}
+
+div_status div_read_device_status(const void* workspace_dev, void* cuda_stream, int32_t* out_status) {
+    if (!workspace_dev || !out_status) return DIV_ERR_NULL;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int32_t v = 0;
+    if (cudaMemcpyAsync(&v, workspace_dev, sizeof(v), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return DIV_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return DIV_ERR_CUDA;
+    *out_status = v;
+    return DIV_OK;
+}
+
+}  // extern "C"

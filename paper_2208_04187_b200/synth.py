@@ -8,7 +8,7 @@ them: same shapes, post-ReLU sparsity (about half the values exactly zero), a sp
 smooth component a few pixels wide (so that the block mean carries real signal) and pixel
 noise on top.
 
-Recipe (all draws from numpy.random.Generator(PCG64(data_seed)), fp32):
+Recipe (sample n of a tensor draws from numpy.random.Generator(PCG64([data_seed, n])), fp32):
   eps  iid N(0,1) per element
   g    smooth field: iid N(0,1) on a (ceil(H/4)+1) x (ceil(W/4)+1) lattice per (n,c) plane,
        bilinearly interpolated to H x W (4-pixel correlation length)
@@ -67,27 +67,34 @@ def _interp_matrix(out_len: int, lattice_len: int) -> np.ndarray:
     return m
 
 
-def smooth_field(rng: np.random.Generator, n: int, c: int, h: int, w: int) -> np.ndarray:
+def smooth_field(rng: np.random.Generator, c: int, h: int, w: int) -> np.ndarray:
     hl = -(-h // CORRELATION_PX) + 1
     wl = -(-w // CORRELATION_PX) + 1
-    lattice = rng.standard_normal((n * c, hl, wl), dtype=np.float32)
+    lattice = rng.standard_normal((c, hl, wl), dtype=np.float32)
     mh = _interp_matrix(h, hl)
     mw = _interp_matrix(w, wl)
-    field = np.matmul(np.matmul(mh[None], lattice), mw.T[None])
-    return field.reshape(n, c, h, w)
+    return np.matmul(np.matmul(mh[None], lattice), mw.T[None])
+
+
+def sample_map(c: int, h: int, w: int, kind: str, data_seed: int, n: int) -> np.ndarray:
+    """Sample `n` (shape C x H x W, fp32) of the tensor with this data_seed; samples are seeded one by one."""
+    rng = np.random.Generator(np.random.PCG64([int(data_seed), int(n)]))
+    g = smooth_field(rng, c, h, w)
+    eps = rng.standard_normal((c, h, w), dtype=np.float32)
+    if kind == "bn":
+        return (eps + g).astype(np.float32)
+    if kind == "relu":
+        m = rng.integers(0, 2, size=(c, h, w), dtype=np.uint8).astype(np.float32)
+        return (m * np.abs(g + np.float32(0.1) * eps)).astype(np.float32)
+    raise ValueError(f"unknown kind {kind!r}")
 
 
 def activation_map(n: int, c: int, h: int, w: int, kind: str, data_seed: int) -> np.ndarray:
     """One fp32 N x C x H x W activation map of the given kind ("relu" or "bn")."""
-    rng = np.random.Generator(np.random.PCG64(data_seed))
-    g = smooth_field(rng, n, c, h, w)
-    eps = rng.standard_normal((n, c, h, w), dtype=np.float32)
-    if kind == "bn":
-        return (eps + g).astype(np.float32)
-    if kind == "relu":
-        m = rng.integers(0, 2, size=(n, c, h, w), dtype=np.uint8).astype(np.float32)
-        return (m * np.abs(g + np.float32(0.1) * eps)).astype(np.float32)
-    raise ValueError(f"unknown kind {kind!r}")
+    out = np.empty((n, c, h, w), dtype=np.float32)
+    for i in range(n):
+        out[i] = sample_map(c, h, w, kind, data_seed, i)
+    return out
 
 
 def to_bf16_bits(x32: np.ndarray) -> np.ndarray:
@@ -99,6 +106,12 @@ def to_bf16_bits(x32: np.ndarray) -> np.ndarray:
 def make_input(spec: TensorSpec) -> np.ndarray:
     """The tensor of `spec`: float32 array, or uint16 bfloat16 bit patterns for bf16 specs."""
     x = activation_map(spec.n, spec.c, spec.h, spec.w, spec.kind, spec.data_seed)
+    return to_bf16_bits(x) if spec.x_dtype == "bf16" else x
+
+
+def make_sample(spec: TensorSpec, n: int) -> np.ndarray:
+    """Sample `n` of the tensor of `spec` with a leading axis of 1 (same bits as make_input(spec)[n:n+1])."""
+    x = sample_map(spec.c, spec.h, spec.w, spec.kind, spec.data_seed, n)[None]
     return to_bf16_bits(x) if spec.x_dtype == "bf16" else x
 
 
