@@ -89,7 +89,8 @@ typedef struct div_layout {
 
 /* How div_compress will run a descriptor (introspection for tests and benchmarks). */
 typedef struct div_plan {
-    int32_t fused;          /* 1: single fused pass over x;  0: two-pass general kernels      */
+    int32_t fused;          /* 2: fused single pass, strip kernel (W%4==0, B in {4,8}, Q in {2,4,8});
+                               1: fused single pass, general kernel;  0: two-pass general kernels */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
     int32_t stages;         /* shared-memory ring depth (fused only)                          */
@@ -102,7 +103,8 @@ typedef struct div_plan {
 } div_plan;
 
 /* flags of div_compress_ex */
-#define DIV_FLAG_FORCE_TWO_PASS 1u   /* never take the fused kernel */
+#define DIV_FLAG_FORCE_TWO_PASS 1u   /* never take a fused kernel                          */
+#define DIV_FLAG_NO_STRIP_KERNEL 2u  /* never take the strip variant of the fused kernel   */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:

@@ -16,6 +16,7 @@ DIV_OK = 0
 DIV_ERR_NULL, DIV_ERR_SHAPE, DIV_ERR_PARAM, DIV_ERR_ALIGN, DIV_ERR_CAPACITY, DIV_ERR_CUDA, DIV_ERR_TIMEOUT = range(1, 8)
 DIV_F32, DIV_BF16 = 0, 1
 DIV_FLAG_FORCE_TWO_PASS = 1
+DIV_FLAG_NO_STRIP_KERNEL = 2
 DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 
 EXPORTED_SYMBOLS = (

@@ -8,6 +8,7 @@
 #include "common.cuh"
 #include "decompress.cuh"
 #include "fused.cuh"
+#include "fused_v.cuh"
 #include "twopass.cuh"
 
 namespace {
@@ -16,6 +17,7 @@ using namespace divk;
 typedef __nv_bfloat16 bf16;
 
 constexpr uint64_t SECTION_ALIGN = 128;
+constexpr uint32_t DIV_FLAG_ALL = DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL;
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
@@ -167,13 +169,23 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     if (!desc || !out) return DIV_ERR_NULL;
     const div_status st = check_desc(desc);
     if (st != DIV_OK) return st;
-    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    if (flags & ~DIV_FLAG_ALL) return DIV_ERR_PARAM;
     const Shape s = make_shape(desc);
     *out = div_plan();
     FusedPlan fp;
-    const bool fused = !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
-    out->fused = fused ? 1 : 0;
-    if (fused) {
+    VPlan vp;
+    const bool vec = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
+    const bool fused = !vec && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
+    out->fused = vec ? 2 : (fused ? 1 : 0);
+    if (vec) {
+        out->grid = vp.grid;
+        out->threads = vp.threads;
+        out->stages = vp.stages;
+        out->lag = vp.lag;
+        out->smem_bytes = vp.smem_bytes;
+        out->chunk_elems = vp.chunk_elems;
+        out->chunks_per_sample = vp.chunks_per_sample;
+    } else if (fused) {
         out->grid = fp.grid;
         out->threads = fp.threads;
         out->stages = fp.stages;
@@ -195,7 +207,7 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if (!desc || !x_dev || !comp_dev || !workspace_dev) return DIV_ERR_NULL;
     div_status st = check_desc(desc);
     if (st != DIV_OK) return st;
-    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    if (flags & ~DIV_FLAG_ALL) return DIV_ERR_PARAM;
     if (!aligned16(x_dev) || !aligned16(comp_dev) || !aligned16(workspace_dev)) return DIV_ERR_ALIGN;
     const Shape s = make_shape(desc);
     div_layout lo;
@@ -205,6 +217,10 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
     uint8_t* blob = (uint8_t*)comp_dev;
     uint32_t* ws = (uint32_t*)workspace_dev;
+    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL))) {
+        VPlan vp;
+        if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream);
+    }
     if (!(flags & DIV_FLAG_FORCE_TWO_PASS)) {
         FusedPlan fp;
         if (plan_fused(desc, s, &fp) == DIV_OK) return compress_fused(desc, s, lo, fp, x_dev, blob, ws, seed, stream);

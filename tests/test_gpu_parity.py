@@ -16,6 +16,7 @@ from paper_2208_04187_b200 import binding, build, synth
 pytestmark = pytest.mark.gpu
 
 TWO_PASS = binding.DIV_FLAG_FORCE_TWO_PASS
+NO_STRIP = binding.DIV_FLAG_NO_STRIP_KERNEL
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -107,7 +108,7 @@ def small_input(n, c, h, w, x_dtype, seed):
 
 
 @pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(map(str, c)))
-@pytest.mark.parametrize("flags", [0, TWO_PASS], ids=["default", "two_pass"])
+@pytest.mark.parametrize("flags", [0, NO_STRIP, TWO_PASS], ids=["default", "general_fused", "two_pass"])
 def test_small_cases_match_the_checker(case, flags):
     n, c, h, w, block, q, xd, ld = case
     x = small_input(n, c, h, w, xd, seed=n + c + h + w + block + q)
@@ -117,15 +118,21 @@ def test_small_cases_match_the_checker(case, flags):
 def test_fused_path_is_taken_where_expected():
     """Guards against silently testing only the general kernels."""
     fused = {case: binding.div_plan_query(binding.make_desc(*case)).fused for case in SMALL}
-    assert fused[(3, 4, 32, 32, 8, 2, "f32", "f32")] == 1
+    assert fused[(3, 4, 32, 32, 8, 2, "f32", "f32")] == 2
+    assert fused[(2, 4, 32, 32, 4, 2, "f32", "f32")] == 2
+    assert fused[(2, 4, 28, 28, 8, 2, "f32", "bf16")] == 2
+    assert fused[(2, 8, 32, 32, 8, 2, "bf16", "bf16")] == 2
+    assert fused[(2, 8, 16, 16, 4, 4, "bf16", "bf16")] == 2
+    assert fused[(2, 4, 32, 32, 8, 1, "f32", "f32")] == 1          # Q = 1: general fused kernel
     assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 1
     assert fused[(2, 16, 7, 7, 8, 2, "f32", "f32")] == 1
-    assert fused[(2, 8, 32, 32, 8, 2, "bf16", "bf16")] == 1
+    assert fused[(2, 3, 40, 24, 16, 2, "f32", "f32")] == 1
+    assert binding.div_plan_query(binding.make_desc(3, 4, 32, 32, 8, 2), NO_STRIP).fused == 1
     assert fused[(1, 2, 3, 3, 2, 2, "f32", "f32")] == 0          # sample is not a whole number of words
     assert fused[(2, 2, 70, 70, 64, 2, "f32", "f32")] == 0        # block wider than a warp
     for spec in synth.config2() + synth.config1() + synth.config3():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
-        assert binding.div_plan_query(d).fused == 1, spec.label()
+        assert binding.div_plan_query(d).fused == (2 if spec.w % 4 == 0 else 1), spec.label()
         assert binding.div_plan_query(d).decompress_fast == (1 if spec.w % 4 == 0 else 0)
 
 
@@ -182,7 +189,7 @@ def test_guard_bands_stay_untouched():
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
                  (2, 8, 32, 32, 8, 2, "bf16", "bf16")]:
         n, c, h, w, block, q, xd, ld = case
-        for flags in (0, TWO_PASS):
+        for flags in (0, NO_STRIP, TWO_PASS):
             x = small_input(n, c, h, w, xd, seed=7)
             codec = binding.Codec(n, c, h, w, block, q, xd, ld)
             pad = 4096
@@ -235,7 +242,7 @@ def assert_sampled_parity(spec, seed, sample_ids, flags=0):
 def test_config0_full():
     spec = synth.config0()[0]
     x = synth.make_input(spec)
-    for flags in (0, TWO_PASS):
+    for flags in (0, NO_STRIP, TWO_PASS):
         assert_full_parity(x, spec.block, spec.qbits, 0, flags=flags)
 
 
@@ -250,8 +257,9 @@ def test_config2_resnet50_imagenet(spec):
     assert_sampled_parity(spec, 0, [0, 31, 63])
 
 
-def test_config2_two_pass_on_one_tensor():
+def test_config2_other_paths_on_one_tensor():
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=TWO_PASS)
+    assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=NO_STRIP)
 
 
 @pytest.mark.parametrize("spec", synth.config3(), ids=lambda s: s.label())
