@@ -2,8 +2,8 @@
 """Benchmark of the DIVISION compress / decompress pair on B200.
 
 One "step" = one pass of the whole hot path over the ResNet-50 / ImageNet-shaped activation set
-(batch 64, fp32, B = 8, Q = 2; five maps): every map is compressed (Algorithm 1 lines 3-6), then
-every map is decompressed (lines 10-11).
+(batch 64, fp32, B = 8, Q = 2; five maps): every map is compressed (Algorithm 1, forward loop), then
+every map is decompressed (Algorithm 1, backward loop).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 

@@ -3,7 +3,7 @@
  *
  * The operation is the per-layer pair of DIVISION ("Memory Efficient Training via Dual
  * Activation Precision"), Sec. 4.1 "Activation Map Compression" and Sec. 4.2 "Activation Map
- * Decompression" (Algorithm 1, lines 3-6 and 10-11):
+ * Decompression" (Algorithm 1, forward and backward loops):
  *
  *   compress    H^L = AveragePooling(H), window = stride = B                    (Sec. 4.1)
  *               H^H = H - UpSampling(H^L), nearest interpolation                (Sec. 4.1)
@@ -115,7 +115,7 @@ typedef struct div_plan {
 div_status div_compressed_bytes(const div_desc* desc, div_layout* out);
 
 /*
- * Compress one activation map (Sec. 4.1; Algorithm 1 lines 3-6).
+ * Compress one activation map (Sec. 4.1; Algorithm 1, forward loop).
  *   desc           host; the problem statement
  *   x_dev          device; N*C*H*W values of x_dtype, contiguous NCHW; read only
  *   comp_dev       device; receives the blob; at least layout.total_bytes
@@ -137,7 +137,7 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
                            uint32_t flags);
 
 /*
- * Decompress (Sec. 4.2; Algorithm 1 lines 10-11): x_hat = UpSampling(H^L) + Delta*V^H + delta,
+ * Decompress (Sec. 4.2; Algorithm 1, backward loop): x_hat = UpSampling(H^L) + Delta*V^H + delta,
  * rounded to x_dtype.
  *   comp_dev    device; a blob written by div_compress with the SAME desc; read only
  *   comp_bytes  bytes valid at comp_dev (>= layout.total_bytes)

@@ -10,7 +10,7 @@ separately from the same written definitions (the paper for the method; the "for
 notes below for what the paper leaves open).
 
 What the method computes (DIVISION, Sec. 4.1 "Activation Map Compression" and Sec. 4.2
-"Activation Map Decompression"; Algorithm 1 lines 3-6 and 10-11):
+"Activation Map Decompression"; the forward and backward loops of Algorithm 1):
 
   compress    H^L = AveragePooling(H)            window = stride = B           (Sec. 4.1)
               H^H = H - UpSampling(H^L)          nearest interpolation         (Sec. 4.1)
@@ -333,7 +333,7 @@ class Compressed:
 
 def compress(x: np.ndarray, block: int, qbits: int, seed: int,
              x_dtype: str = F32, lfc_dtype: str = F32, first_sample: int = 0) -> Compressed:
-    """Algorithm 1 lines 3-6 for one activation map H of shape N x C x H x W.
+    """Forward-loop steps of Algorithm 1 (pooling, residual, Quant, cache) for one activation map H of shape N x C x H x W.
 
     `first_sample`: x holds samples first_sample, first_sample+1, ... of a larger mini-batch (samples
     are independent, so a slice of a batch can be checked alone; only the random stream depends on
@@ -344,13 +344,13 @@ def compress(x: np.ndarray, block: int, qbits: int, seed: int,
     x32 = widen_input(x, x_dtype)
     n, c, h, w = x32.shape
     chw = c * h * w
-    lfc = round_to_dtype(lfc_mean_f32(x32, block), lfc_dtype)           # line 3 (+ storage rounding)
-    r = (x32 - upsample_nearest(lfc, block, h, w)).reshape(n, chw)       # line 4, one fp32 rounding
+    lfc = round_to_dtype(lfc_mean_f32(x32, block), lfc_dtype)           # AveragePooling (+ storage rounding)
+    r = (x32 - upsample_nearest(lfc, block, h, w)).reshape(n, chw)       # residual, one fp32 rounding
     codes = np.empty((n, chw), dtype=np.uint8)
     delta = np.empty(n, dtype=np.float32)
     step = np.empty(n, dtype=np.float32)
     e = np.arange(chw, dtype=np.uint64)
-    for i in range(n):                                                   # line 5, per sample
+    for i in range(n):                                                   # Quant, per sample
         delta[i], step[i], scale = sample_stats(r[i], qbits)
         codes[i] = quantize(r[i], delta[i], scale, divrng_fields(seed, first_sample + i, e), qbits)
     words = pack_codes(codes.reshape(-1), qbits)
@@ -359,7 +359,7 @@ def compress(x: np.ndarray, block: int, qbits: int, seed: int,
 
 
 def decompress(comp: Compressed) -> np.ndarray:
-    """Algorithm 1 lines 10-11; returns fp32 values, already rounded to the activation dtype."""
+    """Backward-loop steps of Algorithm 1 (Dequant, up-sample and add); returns fp32 values, already rounded to the activation dtype."""
     n, c, h, w = comp.shape
     codes = unpack_codes(comp.words, comp.qbits, n * c * h * w).reshape(n, c * h * w)
     hh = np.empty((n, c * h * w), dtype=np.float32)

@@ -15,13 +15,14 @@ namespace divk {
 // workspace layout (device scratch owned by the caller)
 //   word 0          : device status (0 = ok, 7 = a bounded wait ran out)
 //   word 1          : detail of the first failure (sample index)
-//   words 16 + 8n.. : per-sample slot { ~key(min), key(max), arrivals, unused,
-//                                        64-bit parameter word (fused kernel), unused, unused }
+//   words 16 + 32n.. : per-sample slot of 128 bytes (one cache line each, so that the slots of
+//                      neighbouring samples do not share an L2 line): { ~key(min), key(max), arrivals,
+//                      unused, 64-bit parameter word (general fused kernel), unused ... }
 // key() maps a float to an unsigned integer with the same ordering, so that integer atomicMax
 // implements float max (and, on the complemented key, float min).  All-zero is the neutral state.
 // ---------------------------------------------------------------------------------------------
 constexpr int WS_HEADER_WORDS = 16;
-constexpr int WS_SLOT_WORDS = 8;
+constexpr int WS_SLOT_WORDS = 32;
 
 __device__ __forceinline__ uint32_t float_key(float f) {
     uint32_t b = __float_as_uint(f);

@@ -1,4 +1,4 @@
-// Decompress kernels (DIVISION Sec. 4.2, Eq. 10; Algorithm 1 lines 10-11):
+// Decompress kernels (DIVISION Sec. 4.2, Eq. 10; Algorithm 1, backward loop):
 //   x_hat = UpSampling(H^L) + (Delta * V^H + delta), rounded to the activation dtype.
 // One fused pass: unpack, dequantise, add the nearest-upsampled low-frequency value, store.
 #pragma once

@@ -1,4 +1,4 @@
-// Fused single-pass compress kernel (DIVISION Sec. 4.1; Algorithm 1 lines 3-6) for sm_100a.
+// Fused single-pass compress kernel (DIVISION Sec. 4.1; Algorithm 1, forward loop) for sm_100a.
 //
 // x is read from HBM exactly once.  The per-sample min / max of the residual is a dependency that
 // spans the whole sample, so the residuals wait ON CHIP between the two halves of the work:

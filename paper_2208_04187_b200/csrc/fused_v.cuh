@@ -1,37 +1,53 @@
-// Vectorised fused single-pass compress kernel (DIVISION Sec. 4.1; Algorithm 1 lines 3-6) for the
+// Vectorised fused single-pass compress kernel (DIVISION Sec. 4.1; Algorithm 1, forward loop) for the
 // common CNN shapes: W % 4 == 0, B in {4, 8}, Q in {2, 4, 8}.
 //
-// Same plan as the general fused kernel (fused.cuh): x is read from HBM once, each chunk waits in a
-// shared-memory ring between the "reduce" half (block means, residual extremes) and the "quantise"
-// half (Eq. 9 with stochastic rounding, packing), and the per-sample (delta, scale) travel through a
-// slot in global scratch.  What differs is the work decomposition, chosen for instruction count:
+// x is read from HBM once.  Each chunk waits in a shared-memory ring between the "reduce" half (block
+// means, residual extremes) and the "quantise" half (Eq. 9 with stochastic rounding, packing), because
+// the per-sample (delta, scale) are only known once every CTA has reduced its share of the sample.
 //
-//   * a STRIP is 4 adjacent columns of one tile row band (4 x B elements); one thread owns a strip:
-//     B 16-byte shared-memory loads, the column sums of its 4 columns in registers, one shuffle to
-//     meet the other half of a B = 8 tile.  No predicates and no index arithmetic per element;
-//   * a UNIT is 32 consecutive strips (one per lane).  Units are dealt round-robin to the consumer
-//     warps; warp w runs the reduce half of unit w + i*NW and then the quantise half of the unit
-//     `lag` positions earlier, so the wait for the sample's parameters is normally already over;
-//   * the quantise half re-reads x from shared memory, subtracts the stored low-frequency value
-//     (kept per strip in shared memory) and emits the 4 codes of each strip row as one byte (Q = 2),
-//     half-word (Q = 4) or word (Q = 8) straight to the packed stream: lanes of a warp write
-//     consecutive bytes.
+// Roles inside a CTA (one CTA per SM, persistent):
+//   warp 0   producer: one lane streams the chunks into the ring with bulk asynchronous copies;
+//   warp 1   watcher: one lane waits, per chunk, until the chunk's sample is complete grid-wide (it
+//            polls the sample's arrival counter in global scratch, slowly, so that the counter's L2
+//            slice is not flooded), derives (delta, scale) and posts them in shared memory;
+//   others   workers.  Work is cut into UNITS of 32 strips (a strip = 4 adjacent columns of one tile
+//            row band, 4 x B elements, owned by one lane: B 16-byte shared-memory loads, column sums
+//            in registers, one shuffle to meet the other half of a B = 8 tile).  Units are dealt
+//            round-robin to the worker warps.  Each warp keeps two cursors, "next unit to reduce" and
+//            "next unit to quantise", and always does whichever is possible, quantising first: nobody
+//            blocks on the grid-wide dependency while loaded chunks are waiting to be reduced, so the
+//            whole ring is available to hide that dependency's latency.
+//   * the reduce half leaves, per strip, a 16-byte record in shared memory (stored low-frequency value,
+//     where the strip sits in the stage, its index in the sample, its in-bounds rows); the quantise
+//     half re-reads x from shared memory, subtracts the stored low-frequency value and emits the 4
+//     codes of each strip row as one byte (Q = 2), half-word (Q = 4) or word (Q = 8) straight to the
+//     packed stream: lanes of a warp write consecutive bytes.  Its fp32 arithmetic runs on packed
+//     pairs (add/sub/mul/fma .f32x2: two IEEE results per instruction, same roundings as the scalar
+//     forms).
 //   * chunks are runs of `cb` consecutive tile row bands of one sample (they may cross planes);
-//     chunk j goes to CTA j mod gridDim.x.
+//     chunk j goes to CTA j mod gridDim.x, so the CTAs sweep the samples together.
 //
-// All waits are bounded exactly as in fused.cuh.
+// Every wait is bounded: when a limit runs out the kernel records DIV_ERR_TIMEOUT in the workspace
+// status word, stops waiting everywhere, lets its own copies land and returns.  The launch is
+// cooperative only to be certain that all CTAs are resident (no grid-wide barrier is used).
 #pragma once
 
 #include "fused.cuh"
 
 namespace divk {
 
-#ifndef DIVK_V_CONSUMER_WARPS
-#define DIVK_V_CONSUMER_WARPS 16
+#ifndef DIVK_V_WORKER_WARPS
+#define DIVK_V_WORKER_WARPS 22
 #endif
-constexpr int V_CONSUMER_WARPS = DIVK_V_CONSUMER_WARPS;
-constexpr int V_THREADS = 32 * (1 + V_CONSUMER_WARPS);
-constexpr int V_MAX_STAGES = 8;
+#ifndef DIVK_V_TARGET_BYTES
+#define DIVK_V_TARGET_BYTES (32 * 1024)
+#endif
+#ifndef DIVK_V_POLL_NS
+#define DIVK_V_POLL_NS 200
+#endif
+constexpr int V_WORKER_WARPS = DIVK_V_WORKER_WARPS;
+constexpr int V_THREADS = 32 * (2 + V_WORKER_WARPS);
+constexpr int V_MAX_STAGES = 16;
 
 struct VPlan {
     int32_t grid, threads, stages, lag, smem_bytes;
@@ -57,6 +73,8 @@ struct VParams {
     uint64_t seed;
     uint64_t total_chunks;
     uint32_t expected_arrivals;
+    uint32_t last_slots;          // strip slots of a sample's last (possibly short) chunk
+    uint64_t rng_row_step;        // counter increment of the random stream from one row to the next (K_GROUP * W/4)
     uint64_t timeout_ns;
 };
 
@@ -64,13 +82,27 @@ struct VDesc {
     uint32_t n, e0, bi0, nslots;
 };
 
+// per-stage descriptor, written by the producer before it issues the stage's copy
+struct VStage {
+    uint32_t n;          // sample
+    uint32_t e0;         // in-sample index of the chunk's first element
+    uint32_t bi0;        // first band
+    uint32_t nslots;     // strip slots of the chunk
+};
+
 struct VCtl {
-    uint64_t full[V_MAX_STAGES];
-    uint64_t empty[V_MAX_STAGES];
-    uint32_t kmin[V_MAX_STAGES];
+    uint64_t full[V_MAX_STAGES];        // producer -> workers: chunk landed
+    uint64_t empty[V_MAX_STAGES];       // workers -> producer: stage may be overwritten
+    uint32_t issued[V_MAX_STAGES];      // 1 + index of the chunk whose copy was last issued into the stage
+    uint32_t reduced[V_MAX_STAGES];     // 1 + index of the chunk whose reduce half is complete in this CTA
+    uint32_t posted[V_MAX_STAGES];      // 1 + index of the chunk whose (delta, scale) are posted below
+    float par_delta[V_MAX_STAGES];
+    float par_scale[V_MAX_STAGES];
+    uint32_t kmin[V_MAX_STAGES];        // ~key(min r), key(max r) folded over the units of the chunk
     uint32_t kmax[V_MAX_STAGES];
-    uint32_t done1[V_MAX_STAGES];
-    uint32_t done2[V_MAX_STAGES];
+    uint32_t done1[V_MAX_STAGES];       // units of the chunk that finished the reduce half
+    uint32_t done2[V_MAX_STAGES];       // units of the chunk that finished the quantise half
+    VStage desc[V_MAX_STAGES];
     uint32_t failed;
 };
 
@@ -110,10 +142,17 @@ __device__ __forceinline__ uint32_t atom_add_acq_rel(uint32_t* p, uint32_t v) {
 __device__ __forceinline__ void red_max_relaxed(uint32_t* p, uint32_t v) {
     asm volatile("red.relaxed.gpu.global.max.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_volatile(const uint32_t* p) { return *(const volatile uint32_t*)p; }
+__device__ __forceinline__ void sts_volatile(uint32_t* p, uint32_t v) { *(volatile uint32_t*)p = v; }
 
 // bounded waits (same policy as fused.cuh, on this kernel's control block)
 __device__ __forceinline__ bool v_give_up(const VParams& p, VCtl* ctl, uint64_t& t0) {
-    if (*(volatile uint32_t*)&ctl->failed || ld_relaxed_u32(p.ws) != 0u) return true;
+    if (lds_volatile(&ctl->failed) || ld_relaxed_u32(p.ws) != 0u) return true;
     const uint64_t t = now_ns();
     if (t0 == 0) t0 = t;
     return t - t0 > p.timeout_ns;
@@ -121,7 +160,7 @@ __device__ __forceinline__ bool v_give_up(const VParams& p, VCtl* ctl, uint64_t&
 __device__ __forceinline__ void v_record_failure(const VParams& p, VCtl* ctl, uint32_t detail) {
     atomicCAS(p.ws, 0u, (uint32_t)DIV_ERR_TIMEOUT);
     atomicCAS(p.ws + 1, 0u, detail);
-    *(volatile uint32_t*)&ctl->failed = 1u;
+    sts_volatile(&ctl->failed, 1u);
 }
 __device__ __forceinline__ bool v_wait_barrier(uint64_t* bar, uint32_t parity, const VParams& p, VCtl* ctl) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -136,51 +175,134 @@ __device__ __forceinline__ bool v_wait_barrier(uint64_t* bar, uint32_t parity, c
     return true;
 }
 
-// 4 adjacent values of a staged strip row, widened to fp32
-template <typename XT> struct StripRow;
-template <> struct StripRow<float> {
-    static __device__ __forceinline__ float4 load(const float* p) { return *reinterpret_cast<const float4*>(p); }
-};
-template <> struct StripRow<__nv_bfloat16> {
-    static __device__ __forceinline__ float4 load(const __nv_bfloat16* p) {
-        const uint2 u = *reinterpret_cast<const uint2*>(p);
-        return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
-                           __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u));
-    }
-};
-
 template <int Q> struct PackedUnit;
 template <> struct PackedUnit<2> { typedef uint8_t type; };
 template <> struct PackedUnit<4> { typedef uint16_t type; };
 template <> struct PackedUnit<8> { typedef uint32_t type; };
 
-// geometry of the strip a lane owns inside a chunk
-struct Strip {
-    uint32_t off;     // element offset of its first element inside the staged chunk
-    uint32_t e;       // the same as in-sample flat index
-    uint32_t rows;    // in-bounds rows of its band
-    uint32_t ts;      // tile index inside the sample (plane * TPP + bh * Wb + bw)
-    uint32_t q;       // slot inside the band
-    bool ok;          // slot holds real columns
+// ------------------------------------------------------------------------------------------------
+// packed fp32 pairs (one instruction works on two values; IEEE, one rounding per value)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t pk2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ uint64_t pk2u(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void upk2u(uint64_t v, uint32_t& lo, uint32_t& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t add2_rn(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2_rp(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rp.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t sub2_rn(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul2_rn(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2_rn(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+// a staged strip row as two packed pairs (x, y) and (z, w), widened to fp32
+template <typename XT> struct StripRow2;
+template <> struct StripRow2<float> {
+    static __device__ __forceinline__ void load(const unsigned char* p, uint64_t& xy, uint64_t& zw) {
+        const ulonglong2 v = *reinterpret_cast<const ulonglong2*>(p);
+        xy = v.x;
+        zw = v.y;
+    }
 };
-template <int P2>
-__device__ __forceinline__ Strip strip_of(const VParams& p, const VDesc& d, uint32_t sl) {
-    constexpr uint32_t LPT = P2 / 4;
-    const Shape& s = p.s;
-    Strip t;
-    const uint32_t slc = sl < d.nslots ? sl : 0u;
-    const uint32_t band_local = fdiv(slc, p.by_spb);
-    t.q = slc - band_local * p.pl.spb;
-    const uint32_t bi = d.bi0 + band_local;
-    const uint32_t plane = fdiv(bi, p.by_hb);
-    const uint32_t bh = bi - plane * s.Hb;
-    t.rows = min(s.B, s.H - bh * s.B);
-    const uint32_t col0 = 4u * t.q;
-    t.ok = (sl < d.nslots) && (col0 < s.W);
-    t.e = plane * s.HW + bh * s.B * s.W + (t.ok ? col0 : 0u);
-    t.off = t.e - d.e0;
-    t.ts = plane * s.TPP + bh * s.Wb + t.q / LPT;
-    return t;
+template <> struct StripRow2<__nv_bfloat16> {
+    static __device__ __forceinline__ void load(const unsigned char* p, uint64_t& xy, uint64_t& zw) {
+        const uint2 u = *reinterpret_cast<const uint2*>(p);
+        xy = pk2u(u.x << 16, u.x & 0xFFFF0000u);
+        zw = pk2u(u.y << 16, u.y & 0xFFFF0000u);
+    }
+};
+
+// Codes of two elements sharing the 32-bit half `h` of a random word (Eq. 9 with stochastic
+// rounding), same arithmetic as quant_bits(): returns the two results MAGIC_CEIL_BITS + code.
+__device__ __forceinline__ void quant2(uint64_t x01, uint64_t stored2, uint64_t delta2, uint64_t scale2, float qmax,
+                                       uint32_t h, uint32_t& b0, uint32_t& b1) {
+    const uint64_t t01 = mul2_rn(sub2_rn(sub2_rn(x01, stored2), delta2), scale2);
+    float t0, t1;
+    upk2(t01, t0, t1);
+    t0 = fminf(t0, qmax);
+    t1 = fminf(t1, qmax);
+    // 2^23 + field as a float: the 16-bit field in the low mantissa bits
+    const uint64_t f01 = sub2_rn(pk2u(__byte_perm(h, 0x4B000000u, 0x7610), __byte_perm(h, 0x4B000000u, 0x7632)),
+                                 pk2(8388608.0f, 8388608.0f));                                       // exact
+    const uint64_t d01 = fma2_rn(f01, pk2(-1.52587890625e-05f, -1.52587890625e-05f), pk2(t0, t1));   // fl(t - u)
+    upk2u(add2_rp(d01, pk2(MAGIC_CEIL, MAGIC_CEIL)), b0, b1);
+}
+
+// four elements of one strip row -> their codes packed Q bits apart (low bits first)
+template <int Q>
+__device__ __forceinline__ uint32_t quant_row(uint64_t xy, uint64_t zw, uint64_t stored2, uint64_t delta2,
+                                              uint64_t scale2, uint64_t z) {
+    constexpr float qmax = (float)((1 << Q) - 1);
+    uint32_t b0, b1, b2, b3;
+    quant2(xy, stored2, delta2, scale2, qmax, (uint32_t)z, b0, b1);
+    quant2(zw, stored2, delta2, scale2, qmax, (uint32_t)(z >> 32), b2, b3);
+    constexpr uint32_t BIAS = MAGIC_CEIL_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
+    return b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS;
+}
+
+// the mixing function of the random stream (see rng_group) applied to a prepared counter
+__device__ __forceinline__ uint64_t rng_mix(uint64_t z) {
+    z ^= z >> 32;
+    z *= K_MIX;
+    z ^= z >> 32;
+    z *= K_MIX;
+    z ^= z >> 32;
+    return z;
+}
+
+// per-slot record, written by the reduce half for the quantise half
+//   x: stored low-frequency value (bits)   y: byte offset of the strip inside the stage
+//   z: in-sample index of the strip's first element / 4   w: in-bounds rows (0: the slot is padding)
+
+// position of a worker warp's cursor: unit U of this CTA = unit `u` of the CTA's chunk number `it`
+struct VCursor {
+    uint32_t U, it, u, st, round;
+    bool real;        // the unit holds strips (a short chunk leaves its last unit slots empty)
+};
+__device__ __forceinline__ void v_seek(const VParams& p, VCursor& c, uint32_t U, uint32_t n_units) {
+    c.U = U;
+    if (U >= n_units) {
+        c.real = false;
+        return;
+    }
+    c.it = fdiv(U, p.by_nf);
+    c.u = U - c.it * p.pl.nf;
+    c.round = fdiv(c.it, p.by_K);
+    c.st = c.it - c.round * (uint32_t)p.pl.stages;
+    const uint32_t gc = blockIdx.x + c.it * gridDim.x;
+    const uint32_t k = gc - fdiv(gc, p.by_S) * p.pl.chunks_per_sample;
+    const uint32_t nslots = (k + 1u == p.pl.chunks_per_sample) ? p.last_slots : p.pl.cb * p.pl.spb;
+    c.real = c.u * 32u < nslots;
 }
 
 template <typename XT, typename LT, int Q, int P2>
@@ -193,11 +315,11 @@ fused_v_kernel(const VParams p) {
     const Shape& s = p.s;
     const uint32_t K = p.pl.stages;
     const uint32_t stage_bytes = p.pl.stage_bytes;
-    float* lfcs = reinterpret_cast<float*>(smem + (size_t)K * stage_bytes);
-    VCtl* ctl = reinterpret_cast<VCtl*>(lfcs + (size_t)K * p.pl.slots_per_stage);
+    uint4* recs = reinterpret_cast<uint4*>(smem + (size_t)K * stage_bytes);
+    VCtl* ctl = reinterpret_cast<VCtl*>(recs + (size_t)K * p.pl.slots_per_stage);
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t NW = (blockDim.x >> 5) - 1;
+    const uint32_t NW = (blockDim.x >> 5) - 2;
     const uint32_t G = gridDim.x;
     const uint64_t total = p.total_chunks;
     const uint32_t n_my = blockIdx.x < total ? (uint32_t)((total - blockIdx.x + G - 1) / G) : 0u;
@@ -206,6 +328,9 @@ fused_v_kernel(const VParams p) {
         for (uint32_t i = 0; i < K; ++i) {
             mbar_init(&ctl->full[i], 1);
             mbar_init(&ctl->empty[i], 1);
+            ctl->issued[i] = 0;
+            ctl->reduced[i] = 0;
+            ctl->posted[i] = 0;
             ctl->kmin[i] = 0;
             ctl->kmax[i] = 0;
             ctl->done1[i] = 0;
@@ -219,7 +344,8 @@ fused_v_kernel(const VParams p) {
     if (warp == 0) {
         // ================= producer: one lane streams the chunks into the ring =================
         if (lane == 0) {
-            for (uint32_t it = 0; it < n_my; ++it) {
+            uint32_t it = 0;
+            for (; it < n_my; ++it) {
                 const uint32_t round = fdiv(it, p.by_K);
                 const uint32_t st = it - round * K;
                 if (it >= K && !v_wait_barrier(&ctl->empty[st], (round - 1) & 1, p, ctl)) break;
@@ -227,68 +353,214 @@ fused_v_kernel(const VParams p) {
                 const VDesc d = v_chunk_desc(p, blockIdx.x + it * G, &nelem);
                 const uint32_t bytes = nelem * (uint32_t)sizeof(XT);
                 const XT* src = reinterpret_cast<const XT*>(p.x) + ((size_t)d.n * s.CHW + d.e0);
+                VStage sd;
+                sd.n = d.n;
+                sd.e0 = d.e0;
+                sd.bi0 = d.bi0;
+                sd.nslots = d.nslots;
+                ctl->desc[st] = sd;
                 mbar_arrive_expect_tx(&ctl->full[st], bytes);
                 bulk_load(smem + (size_t)st * stage_bytes, src, bytes, &ctl->full[st]);
+                __threadfence_block();
+                sts_volatile(&ctl->issued[st], it + 1u);
+            }
+            if (it < n_my || lds_volatile(&ctl->failed)) {
+                // a wait gave up somewhere: let the copies still in flight land before the CTA may exit
+                const uint32_t first = it > K ? it - K : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    const uint32_t round = fdiv(j, p.by_K);
+                    uint32_t polls = 0;
+                    while (!mbar_try_wait(&ctl->full[j - round * K], round & 1) && ++polls < (1u << 20)) {
+                    }
+                }
             }
         }
         return;
     }
 
-    // ================= consumers =================
-    const uint32_t cw = warp - 1;
-    const uint32_t nf = p.pl.nf;
-    const uint32_t n_units = n_my * nf;
-    const uint32_t L = (uint32_t)p.pl.lag;
+    if (warp == 1) {
+        // ================= watcher: per chunk, wait for its sample's parameters and post them =================
+        if (lane == 0) {
+            uint32_t have_n = 0xFFFFFFFFu;
+            float delta = 0.f, scale = 0.f;
+            for (uint32_t it = 0; it < n_my; ++it) {
+                const uint32_t round = fdiv(it, p.by_K);
+                const uint32_t st = it - round * K;
+                const VDesc d = v_chunk_desc(p, blockIdx.x + it * G);
+                bool ok = true;
+                if (d.n != have_n) {
+                    uint32_t polls = 0;
+                    uint64_t t0 = 0;
+                    // first the cheap local condition: this CTA's own chunk has been reduced
+                    while (lds_volatile(&ctl->reduced[st]) != it + 1u) {
+                        if ((++polls & 63u) == 0 && v_give_up(p, ctl, t0)) {
+                            ok = false;
+                            break;
+                        }
+                        __nanosleep(40);
+                    }
+                    const uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)d.n * WS_SLOT_WORDS;
+                    polls = 0;
+                    t0 = 0;
+                    while (ok && ld_acquire_u32(slot + 2) != p.expected_arrivals) {
+                        if ((++polls & 7u) == 0 && v_give_up(p, ctl, t0)) {
+                            ok = false;
+                            break;
+                        }
+                        __nanosleep(DIVK_V_POLL_NS);
+                    }
+                    if (!ok) {
+                        v_record_failure(p, ctl, d.n + 1u);
+                        break;
+                    }
+                    const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
+                    delta = qp.delta;
+                    scale = qp.scale;
+                    have_n = d.n;
+                }
+                ctl->par_delta[st] = delta;
+                ctl->par_scale[st] = scale;
+                __threadfence_block();
+                sts_volatile(&ctl->posted[st], it + 1u);
+            }
+        }
+        return;
+    }
+
+    // ================= workers =================
+    const uint32_t cw = warp - 2;
+    const uint32_t n_units = n_my * p.pl.nf;
+    const uint32_t row_bytes = s.W * (uint32_t)sizeof(XT);
+    const uint32_t W4 = s.W >> 2;
     LT* lfc_out = reinterpret_cast<LT*>(p.lfc);
     OutT* packed = reinterpret_cast<OutT*>(p.packed);
-    bool alive = true;
 
-    for (uint32_t U1 = cw; U1 < n_units + L; U1 += NW) {
-        const bool has1 = U1 < n_units;
-        const bool has2 = U1 >= L;
+    VCursor cr, cq;              // next unit to reduce / to quantise
+    v_seek(p, cr, cw, n_units);
+    v_seek(p, cq, cw, n_units);
+    uint32_t idle = 0;
+    uint64_t t0 = 0;
 
-        // ---------------- reduce half of unit U1 ----------------
-        if (has1) {
-            const uint32_t it = fdiv(U1, p.by_nf);
-            const uint32_t u = U1 - it * nf;
-            const uint32_t round = fdiv(it, p.by_K);
-            const uint32_t st = it - round * K;
-            const VDesc d = v_chunk_desc(p, blockIdx.x + it * G);
-            const bool real = u * 32u < d.nslots;      // a short chunk leaves its last unit slots empty
-            if (alive && real) alive = v_wait_barrier(&ctl->full[st], round & 1, p, ctl);
-            if (alive && real) {
-                const uint32_t sl = u * 32u + lane;
-                const Strip t = strip_of<P2>(p, d, sl);
-                const XT* xs = reinterpret_cast<const XT*>(smem + (size_t)st * stage_bytes) + t.off;
-                float4 v[P2];
-                if (__all_sync(0xFFFFFFFFu, t.ok && t.rows == (uint32_t)P2)) {
+    while (cq.U < n_units) {
+        // ---------------- quantise half of the oldest reduced unit, if its parameters are posted ----------------
+        if (cq.U < cr.U) {
+            if (!cq.real) {
+                v_seek(p, cq, cq.U + NW, n_units);
+                continue;
+            }
+            const uint32_t st = cq.st;
+            if (__shfl_sync(0xFFFFFFFFu, lds_volatile(&ctl->posted[st]), 0) == cq.it + 1u) {
+                __threadfence_block();
+                const float delta = ctl->par_delta[st];
+                const float scale = ctl->par_scale[st];
+                const uint32_t n = ctl->desc[st].n;
+                const uint32_t sl = cq.u * 32u + lane;
+                const uint4 rec = recs[(size_t)st * p.pl.slots_per_stage + sl];
+                if (rec.w != 0u) {
+                    const unsigned char* xs = smem + (size_t)st * stage_bytes + rec.y;
+                    const uint64_t stored2 = pk2u(rec.x, rec.x);
+                    const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
+                    uint64_t ctr = rng_sample_base(p.seed, n) + K_GROUP * (uint64_t)(rec.z + 1u);
+                    OutT* out = packed + (((uint64_t)n * s.CHW) >> 2) + rec.z;
+                    if (rec.w == (uint32_t)P2) {
 #pragma unroll
-                    for (int r = 0; r < P2; ++r) v[r] = StripRow<XT>::load(xs + r * s.W);
+                        for (int r = 0; r < P2; ++r) {
+                            uint64_t xy, zw;
+                            StripRow2<XT>::load(xs + r * row_bytes, xy, zw);
+                            out[r * W4] = (OutT)quant_row<Q>(xy, zw, stored2, delta2, scale2, rng_mix(ctr));
+                            ctr += p.rng_row_step;
+                        }
+                    } else {
+                        for (uint32_t r = 0; r < rec.w; ++r) {
+                            uint64_t xy, zw;
+                            StripRow2<XT>::load(xs + r * row_bytes, xy, zw);
+                            out[r * W4] = (OutT)quant_row<Q>(xy, zw, stored2, delta2, scale2, rng_mix(ctr));
+                            ctr += p.rng_row_step;
+                        }
+                    }
+                }
+                // release: the last unit of the chunk hands the stage back to the producer
+                __syncwarp();
+                if (lane == 0) {
+                    const uint32_t units = (ctl->desc[st].nslots + 31u) >> 5;
+                    if (atomicAdd(&ctl->done2[st], 1u) == units - 1u) {
+                        ctl->done2[st] = 0u;
+                        __threadfence_block();
+                        mbar_arrive(&ctl->empty[st]);
+                    }
+                }
+                v_seek(p, cq, cq.U + NW, n_units);
+                idle = 0;
+                t0 = 0;
+                continue;
+            }
+        }
+
+        // ---------------- reduce half of the next unit, if its chunk has landed ----------------
+        if (cr.U < n_units) {
+            if (!cr.real) {
+                v_seek(p, cr, cr.U + NW, n_units);
+                continue;
+            }
+            const uint32_t st = cr.st;
+            bool landed = __shfl_sync(0xFFFFFFFFu, lds_volatile(&ctl->issued[st]), 0) == cr.it + 1u;
+            if (landed) landed = __any_sync(0xFFFFFFFFu, mbar_try_wait(&ctl->full[st], cr.round & 1));
+            if (landed) {
+                const VStage sd = ctl->desc[st];
+                // geometry of this lane's strip
+                const uint32_t sl = cr.u * 32u + lane;
+                const bool valid = sl < sd.nslots;
+                const uint32_t slc = valid ? sl : 0u;
+                const uint32_t band_local = fdiv(slc, p.by_spb);
+                const uint32_t q = slc - band_local * p.pl.spb;
+                const uint32_t bi = sd.bi0 + band_local;
+                const uint32_t plane = fdiv(bi, p.by_hb);
+                const uint32_t bh = bi - plane * s.Hb;
+                const uint32_t rows = min(s.B, s.H - bh * s.B);
+                const uint32_t col0 = 4u * q;
+                const bool ok = valid && col0 < s.W;
+                const uint32_t e = plane * s.HW + bh * s.B * s.W + (ok ? col0 : 0u);
+                const uint32_t off_bytes = (e - sd.e0) * (uint32_t)sizeof(XT);
+                const unsigned char* xs = smem + (size_t)st * stage_bytes + off_bytes;
+
+                uint64_t vxy[P2], vzw[P2];
+                if (__all_sync(0xFFFFFFFFu, ok && rows == (uint32_t)P2)) {
+#pragma unroll
+                    for (int r = 0; r < P2; ++r) StripRow2<XT>::load(xs + r * row_bytes, vxy[r], vzw[r]);
                 } else {
 #pragma unroll
-                    for (int r = 0; r < P2; ++r)
-                        v[r] = (t.ok && (uint32_t)r < t.rows) ? StripRow<XT>::load(xs + r * s.W)
-                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int r = 0; r < P2; ++r) {
+                        if (ok && (uint32_t)r < rows) {
+                            StripRow2<XT>::load(xs + r * row_bytes, vxy[r], vzw[r]);
+                        } else {
+                            vxy[r] = 0ull;
+                            vzw[r] = 0ull;
+                        }
+                    }
                 }
                 // column sums: balanced tree down the rows of each of the 4 columns
-                float4 c[P2];
+                uint64_t cxy[P2], czw[P2];
 #pragma unroll
-                for (int r = 0; r < P2; ++r) c[r] = v[r];
+                for (int r = 0; r < P2; ++r) {
+                    cxy[r] = vxy[r];
+                    czw[r] = vzw[r];
+                }
 #pragma unroll
                 for (int w = P2; w > 1; w >>= 1) {
 #pragma unroll
                     for (int i = 0; i < w / 2; ++i) {
-                        c[i].x = __fadd_rn(c[2 * i].x, c[2 * i + 1].x);
-                        c[i].y = __fadd_rn(c[2 * i].y, c[2 * i + 1].y);
-                        c[i].z = __fadd_rn(c[2 * i].z, c[2 * i + 1].z);
-                        c[i].w = __fadd_rn(c[2 * i].w, c[2 * i + 1].w);
+                        cxy[i] = add2_rn(cxy[2 * i], cxy[2 * i + 1]);
+                        czw[i] = add2_rn(czw[2 * i], czw[2 * i + 1]);
                     }
                 }
-                float sum = __fadd_rn(__fadd_rn(c[0].x, c[0].y), __fadd_rn(c[0].z, c[0].w));
+                float c0, c1, c2, c3;
+                upk2(cxy[0], c0, c1);
+                upk2(czw[0], c2, c3);
+                float sum = __fadd_rn(__fadd_rn(c0, c1), __fadd_rn(c2, c3));
 #pragma unroll
                 for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-                const uint32_t bw = t.q / LPT;
-                const uint32_t cnt = t.rows * min(s.B, s.W - bw * s.B);
+                const uint32_t bw = q / LPT;
+                const uint32_t cnt = rows * min(s.B, s.W - bw * s.B);
                 const float cntf = (float)cnt;
                 float mean;
                 if ((cnt & (cnt - 1)) == 0)
@@ -296,28 +568,23 @@ fused_v_kernel(const VParams p) {
                 else
                     mean = __fdiv_rn(sum, cntf);
                 const float stored = Elem<LT>::round(mean);
-                if (t.ok && (t.q % LPT) == 0) Elem<LT>::store(lfc_out + (size_t)d.n * s.C * s.TPP + t.ts, mean);
-                lfcs[(size_t)st * p.pl.slots_per_stage + sl] = stored;
+                if (ok && (q % LPT) == 0)
+                    Elem<LT>::store(lfc_out + (size_t)sd.n * s.C * s.TPP + (plane * s.TPP + bh * s.Wb + bw), mean);
+                recs[(size_t)st * p.pl.slots_per_stage + sl] =
+                    make_uint4(__float_as_uint(stored), off_bytes, e >> 2, ok ? rows : 0u);
                 // extremes of x over the strip's in-bounds rows; x -> fl(x - stored) is monotone
                 float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-                if (t.ok) {
-                    if (t.rows == (uint32_t)P2) {
+                if (ok) {
 #pragma unroll
-                        for (int r = 0; r < P2; ++r) {
-                            lo = fmin3(lo, v[r].x, v[r].y);
-                            lo = fmin3(lo, v[r].z, v[r].w);
-                            hi = fmax3(hi, v[r].x, v[r].y);
-                            hi = fmax3(hi, v[r].z, v[r].w);
-                        }
-                    } else {
-#pragma unroll
-                        for (int r = 0; r < P2; ++r) {
-                            if ((uint32_t)r < t.rows) {
-                                lo = fmin3(lo, v[r].x, v[r].y);
-                                lo = fmin3(lo, v[r].z, v[r].w);
-                                hi = fmax3(hi, v[r].x, v[r].y);
-                                hi = fmax3(hi, v[r].z, v[r].w);
-                            }
+                    for (int r = 0; r < P2; ++r) {
+                        if (rows == (uint32_t)P2 || (uint32_t)r < rows) {
+                            float a, b, c, d;
+                            upk2(vxy[r], a, b);
+                            upk2(vzw[r], c, d);
+                            lo = fmin3(lo, a, b);
+                            lo = fmin3(lo, c, d);
+                            hi = fmax3(hi, a, b);
+                            hi = fmax3(hi, c, d);
                         }
                     }
                     lo = __fsub_rn(lo, stored);
@@ -330,113 +597,46 @@ fused_v_kernel(const VParams p) {
                     atomicMax(&ctl->kmin[st], kmin);
                     atomicMax(&ctl->kmax[st], kmax);
                     __threadfence_block();
-                    const uint32_t units = (d.nslots + 31u) >> 5;
+                    const uint32_t units = (sd.nslots + 31u) >> 5;
                     if (atomicAdd(&ctl->done1[st], 1u) == units - 1u) {
                         // last unit of this chunk: fold the chunk into its sample's slot
                         __threadfence_block();
                         const uint32_t smin = atomicExch(&ctl->kmin[st], 0u);
                         const uint32_t smax = atomicExch(&ctl->kmax[st], 0u);
                         ctl->done1[st] = 0u;
-                        uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)d.n * WS_SLOT_WORDS;
-                        if (*(volatile uint32_t*)&ctl->failed == 0u) {
+                        uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)sd.n * WS_SLOT_WORDS;
+                        if (lds_volatile(&ctl->failed) == 0u) {
                             red_max_relaxed(slot + 0, smin);
                             red_max_relaxed(slot + 1, smax);
-                            if (atom_add_acq_rel(slot + 2, 1u) == p.expected_arrivals - 1u) {
-                                const float rlo = key_float(~ld_relaxed_u32(slot + 0));
-                                const float rhi = key_float(ld_relaxed_u32(slot + 1));
-                                const QParams qp = make_qparams(rlo, rhi, Q);
-                                p.stats[2 * (size_t)d.n + 0] = qp.delta;
-                                p.stats[2 * (size_t)d.n + 1] = qp.step;
-                                const uint64_t word = ((uint64_t)(__float_as_uint(qp.scale) | 0x80000000u) << 32) |
-                                                      (uint64_t)__float_as_uint(qp.delta);
-                                st_release_u64(reinterpret_cast<uint64_t*>(slot + 4), word);
+                            const uint32_t before = atom_add_acq_rel(slot + 2, 1u);
+                            sts_volatile(&ctl->reduced[st], cr.it + 1u);
+                            if (before == p.expected_arrivals - 1u) {
+                                // the arrival that completes the sample writes its (delta, Delta) to the blob
+                                const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)),
+                                                                key_float(ld_relaxed_u32(slot + 1)), Q);
+                                p.stats[2 * (size_t)sd.n + 0] = qp.delta;
+                                p.stats[2 * (size_t)sd.n + 1] = qp.step;
                             }
                         }
                     }
                 }
+                v_seek(p, cr, cr.U + NW, n_units);
+                idle = 0;
+                t0 = 0;
+                continue;
             }
         }
 
-        // ---------------- quantise half of unit U1 - L ----------------
-        if (has2) {
-            const uint32_t U2 = U1 - L;
-            const uint32_t it = fdiv(U2, p.by_nf);
-            const uint32_t u = U2 - it * nf;
-            const uint32_t round = fdiv(it, p.by_K);
-            const uint32_t st = it - round * K;
-            const VDesc d = v_chunk_desc(p, blockIdx.x + it * G);
-            const bool real = u * 32u < d.nslots;
-            // the chunk landed long ago, but this warp may not have looked at its barrier yet
-            if (alive && real) alive = v_wait_barrier(&ctl->full[st], round & 1, p, ctl);
-            if (real) {
-                uint64_t word = 0;
-                if (alive) {
-                    if (lane == 0) {
-                        const uint64_t* pw =
-                            reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)d.n * WS_SLOT_WORDS + 4);
-                        uint32_t polls = 0;
-                        uint64_t t0 = 0;
-                        while (true) {
-                            word = ld_relaxed_u64(pw);
-                            if (word >> 63) break;
-                            if ((++polls & 63u) == 0) {
-                                if (v_give_up(p, ctl, t0)) {
-                                    v_record_failure(p, ctl, d.n + 1u);
-                                    word = 0;
-                                    break;
-                                }
-                                __nanosleep(32);
-                            }
-                        }
-                        fence_acq_rel_gpu();
-                    }
-                    word = __shfl_sync(0xFFFFFFFFu, word, 0);
-                    alive = (word >> 63) != 0;
-                }
-                if (alive) {
-                    const float delta = __uint_as_float((uint32_t)word);
-                    const float scale = __uint_as_float((uint32_t)(word >> 32) & 0x7FFFFFFFu);
-                    const uint64_t base = rng_sample_base(p.seed, d.n);
-                    const uint32_t sl = u * 32u + lane;
-                    const Strip t = strip_of<P2>(p, d, sl);
-                    if (t.ok) {
-                        const XT* xs = reinterpret_cast<const XT*>(smem + (size_t)st * stage_bytes) + t.off;
-                        const float stored = lfcs[(size_t)st * p.pl.slots_per_stage + sl];
-                        const uint32_t W4 = s.W >> 2;
-                        const uint32_t g0 = t.e >> 2;
-                        OutT* out = packed + (((uint64_t)d.n * s.CHW) >> 2) + g0;
-                        if (t.rows == (uint32_t)P2) {
-#pragma unroll
-                            for (int r = 0; r < P2; ++r) {
-                                const float4 x4 = StripRow<XT>::load(xs + r * s.W);
-                                const uint64_t z = rng_group(base, g0 + r * W4);
-                                out[r * W4] = (OutT)quant4<Q>(__fsub_rn(x4.x, stored), __fsub_rn(x4.y, stored),
-                                                              __fsub_rn(x4.z, stored), __fsub_rn(x4.w, stored), delta,
-                                                              scale, z);
-                            }
-                        } else {
-                            for (uint32_t r = 0; r < t.rows; ++r) {
-                                const float4 x4 = StripRow<XT>::load(xs + r * s.W);
-                                const uint64_t z = rng_group(base, g0 + r * W4);
-                                out[r * W4] = (OutT)quant4<Q>(__fsub_rn(x4.x, stored), __fsub_rn(x4.y, stored),
-                                                              __fsub_rn(x4.z, stored), __fsub_rn(x4.w, stored), delta,
-                                                              scale, z);
-                            }
-                        }
-                    }
-                }
-                // release: the last unit of the chunk hands the stage back to the producer
-                __syncwarp();
-                if (lane == 0) {
-                    const uint32_t units = (d.nslots + 31u) >> 5;
-                    if (atomicAdd(&ctl->done2[st], 1u) == units - 1u) {
-                        ctl->done2[st] = 0u;
-                        __threadfence_block();
-                        mbar_arrive(&ctl->empty[st]);
-                    }
-                }
+        // ---------------- nothing to do right now ----------------
+        if ((++idle & 15u) == 0) {
+            bool stop = false;
+            if (lane == 0) {
+                stop = v_give_up(p, ctl, t0);
+                if (stop) v_record_failure(p, ctl, 0x40000000u | cq.U);
             }
+            if (__any_sync(0xFFFFFFFFu, stop)) break;
         }
+        __nanosleep(100);
     }
 }
 
@@ -460,13 +660,13 @@ inline div_status plan_v(const div_desc* d, const Shape& s, VPlan* out) {
     pl.threads = V_THREADS;
     const uint32_t band_bytes = s.B * s.W * sx;
     const uint32_t budget = (uint32_t)di.smem_optin - 2048u - (uint32_t)sizeof(VCtl);
-    const uint32_t target = 30u * 1024u;                       // chunk bytes we aim for
+    const uint32_t target = DIVK_V_TARGET_BYTES;               // chunk bytes we aim for
     if (band_bytes + 256u > budget / 4) return DIV_ERR_PARAM;
-    // whole units per chunk where the band geometry allows it
+    // bands per chunk: near the target size, a count that fills whole units of 32 strips where possible
     const uint32_t cbq = 32u / gcd_u32(32u, pl.spb);
     uint32_t cb = target / band_bytes;
-    if (cb >= cbq) cb = cb / cbq * cbq;
     if (cb == 0) cb = 1;
+    if (cb >= cbq) cb = cb / cbq * cbq;
     if (cb > pl.bands_per_sample) cb = pl.bands_per_sample;
     pl.cb = cb;
     pl.nf = (cb * pl.spb + 31u) / 32u;
@@ -474,7 +674,7 @@ inline div_status plan_v(const div_desc* d, const Shape& s, VPlan* out) {
     pl.chunk_elems = cb * s.B * s.W;
     pl.chunks_per_sample = (pl.bands_per_sample + cb - 1) / cb;
     pl.stage_bytes = (cb * band_bytes + 127u) & ~127u;
-    const uint32_t per_stage = pl.stage_bytes + pl.slots_per_stage * 4u;
+    const uint32_t per_stage = pl.stage_bytes + pl.slots_per_stage * 16u;
     uint32_t stages = budget / per_stage;
     if (stages > (uint32_t)V_MAX_STAGES) stages = V_MAX_STAGES;
     if (stages < 4) return DIV_ERR_PARAM;
@@ -485,16 +685,11 @@ inline div_status plan_v(const div_desc* d, const Shape& s, VPlan* out) {
     uint64_t grid = (uint64_t)di.sms;
     if (grid > total_chunks) grid = total_chunks;
     pl.grid = (int32_t)grid;
-    // lag (in units): keep two stages for loads in flight and one for the chunk being reduced
-    const int64_t alive_units = (int64_t)(stages - 3) * pl.nf - V_CONSUMER_WARPS;
-    int64_t lag = alive_units;
-    if (lag < (int64_t)pl.nf) lag = pl.nf;
-    // progress guarantee: units of one sample inside one CTA must fit between the two halves
-    const uint64_t span = ((pl.chunks_per_sample + grid - 1) / grid) * pl.nf;
-    if (span > (uint64_t)lag + V_CONSUMER_WARPS) return DIV_ERR_PARAM;
-    // and the ring must hold everything between the oldest lagging unit and the newest reduced unit
-    if ((uint64_t)(lag + V_CONSUMER_WARPS + pl.nf - 1) / pl.nf + 1 > stages) return DIV_ERR_PARAM;
-    pl.lag = (int32_t)lag;
+    // progress guarantee: a sample completes only when every CTA has reduced all of its chunks of that
+    // sample, so those chunks (plus room for the next copy) must fit in a CTA's ring together
+    const uint64_t span = (pl.chunks_per_sample + grid - 1) / grid;
+    if (span + 2 > stages) return DIV_ERR_PARAM;
+    pl.lag = (int32_t)(stages - span);      // chunks the reduce half may run ahead of the quantise half
     *out = pl;
     return DIV_OK;
 }
@@ -548,6 +743,8 @@ inline div_status compress_fused_v(const div_desc* d, const Shape& s, const div_
     prm.seed = seed;
     prm.total_chunks = (uint64_t)pl.chunks_per_sample * s.N;
     prm.expected_arrivals = expected_arrivals ? expected_arrivals : pl.chunks_per_sample;
+    prm.last_slots = (pl.bands_per_sample - (pl.chunks_per_sample - 1u) * pl.cb) * pl.spb;
+    prm.rng_row_step = K_GROUP * (uint64_t)(s.W / 4u);
     prm.timeout_ns = timeout_ns ? timeout_ns : 2000000000ull;
     typedef __nv_bfloat16 bf16;
     if (d->x_dtype == DIV_F32) {
