@@ -89,14 +89,17 @@ typedef struct div_layout {
 
 /* How div_compress will run a descriptor (introspection for tests and benchmarks). */
 typedef struct div_plan {
-    int32_t fused;          /* 2: fused single pass, strip kernel (W%4==0, B in {4,8}, Q in {2,4,8});
-                               1: fused single pass, general kernel;  0: two-pass general kernels */
+    int32_t fused;          /* 3: one launch, x read from HBM once and re-read from L2 a few rounds later
+                                  (W%4==0, B in {4,8}, Q in {2,4,8});
+                               2: one launch, chunks wait in a shared-memory ring (same shapes);
+                               1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
-    int32_t stages;         /* shared-memory ring depth (fused only)                          */
-    int32_t lag;            /* chunks between min/max and quantise of the same chunk (fused)  */
+    int32_t stages;         /* shared-memory ring depth (ring kernels only)                   */
+    int32_t lag;            /* chunks (ring kernels) or rounds (3) between the reduce and the quantise
+                               half of the same data                                           */
     int32_t smem_bytes;     /* dynamic shared memory per CTA                                  */
-    int64_t chunk_elems;    /* elements per full chunk (fused only)                           */
+    int64_t chunk_elems;    /* elements per full chunk (ring kernels) or per round (3)        */
     int64_t chunks_per_sample;
     int32_t decompress_fast;/* 1: vectorised decompress kernel applies                        */
     int32_t reserved;
@@ -104,7 +107,8 @@ typedef struct div_plan {
 
 /* flags of div_compress_ex */
 #define DIV_FLAG_FORCE_TWO_PASS 1u   /* never take a fused kernel                          */
-#define DIV_FLAG_NO_STRIP_KERNEL 2u  /* never take the strip variant of the fused kernel   */
+#define DIV_FLAG_NO_STRIP_KERNEL 2u  /* never take the strip variant of the ring kernel    */
+#define DIV_FLAG_NO_LAGGED_KERNEL 4u /* never take the lagged (L2 re-read) kernel          */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:

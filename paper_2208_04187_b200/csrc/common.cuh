@@ -39,11 +39,15 @@ __device__ __forceinline__ float key_float(uint32_t k) {
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static __device__ __forceinline__ float load(const float* p) { return *p; }
+    static __device__ __forceinline__ float load_cg(const float* p) { return __ldcg(p); }
     static __device__ __forceinline__ void store(float* p, float v) { *p = v; }
     static __device__ __forceinline__ float round(float v) { return v; }
 };
 template <> struct Elem<__nv_bfloat16> {
     static __device__ __forceinline__ float load(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ float load_cg(const __nv_bfloat16* p) {
+        return __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)) << 16);
+    }
     static __device__ __forceinline__ void store(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
     static __device__ __forceinline__ float round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 };
