@@ -89,17 +89,18 @@ typedef struct div_layout {
 
 /* How div_compress will run a descriptor (introspection for tests and benchmarks). */
 typedef struct div_plan {
-    int32_t fused;          /* 3: one launch, x read from HBM once and re-read from L2 a few rounds later
+    int32_t fused;          /* 2: one launch, chunks wait in a shared-memory ring, strip kernel
                                   (W%4==0, B in {4,8}, Q in {2,4,8});
-                               2: one launch, chunks wait in a shared-memory ring (same shapes);
+                               3: one launch, x read from HBM once and re-read from L2 a little later
+                                  (same shapes; taken when the ring cannot hold a sample's share);
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
     int32_t stages;         /* shared-memory ring depth (ring kernels only)                   */
-    int32_t lag;            /* chunks (ring kernels) or rounds (3) between the reduce and the quantise
+    int32_t lag;            /* chunks (ring kernels) or units (3) between the reduce and the quantise
                                half of the same data                                           */
     int32_t smem_bytes;     /* dynamic shared memory per CTA                                  */
-    int64_t chunk_elems;    /* elements per full chunk (ring kernels) or per round (3)        */
+    int64_t chunk_elems;    /* elements per full chunk (ring kernels) or per unit (3)         */
     int64_t chunks_per_sample;
     int32_t decompress_fast;/* 1: vectorised decompress kernel applies                        */
     int32_t reserved;

@@ -176,17 +176,17 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     FusedPlan fp;
     VPlan vp;
     LPlan lp;
-    const bool lag = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
-    const bool vec = !lag && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
+    const bool vec = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
+    const bool lag = !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
     const bool fused = !lag && !vec && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
     out->fused = lag ? 3 : (vec ? 2 : (fused ? 1 : 0));
     if (lag) {
         out->grid = lp.grid;
         out->threads = lp.threads;
         out->stages = 0;
-        out->lag = (int32_t)lp.lag_rounds;
+        out->lag = (int32_t)lp.lag_units;
         out->smem_bytes = 0;
-        out->chunk_elems = (int64_t)lp.grid * L_WARPS * 32 * 4 * s.B;      // elements one round covers
+        out->chunk_elems = (int64_t)32 * lp.bands_per_lane * 4 * s.B;       // elements of one full unit
         out->chunks_per_sample = lp.units_per_sample;
     } else if (vec) {
         out->grid = vp.grid;
@@ -228,13 +228,13 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
     uint8_t* blob = (uint8_t*)comp_dev;
     uint32_t* ws = (uint32_t*)workspace_dev;
-    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL))) {
-        LPlan lp;
-        if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
-    }
     if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL))) {
         VPlan vp;
         if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream);
+    }
+    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL))) {
+        LPlan lp;
+        if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
     }
     if (!(flags & DIV_FLAG_FORCE_TWO_PASS)) {
         FusedPlan fp;
