@@ -142,6 +142,40 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
                            uint32_t flags);
 
 /*
+ * Compress without a caller-supplied workspace.  (The paper has no counterpart: this is a convenience of
+ * this library.)
+ *
+ * Who needs it: code that may not allocate device memory at the point where it compresses.  Examples are
+ * a host callback or a plug-in running inside somebody else's framework whose memory pool it must not
+ * touch, a process whose device memory budget is fully handed out at start-up, or a latency-critical loop
+ * in which a cudaMalloc (which synchronises the device) is not acceptable.  Such a caller still owns x and
+ * the blob, but cannot produce the few kilobytes of scratch div_compress asks for.
+ *
+ * Here the scratch is a fixed array inside the library (128 bytes per sample, for at most
+ * DIV_STATIC_MAX_SAMPLES samples, about 128 KB).  Every GPU that loads the library holds that array until
+ * the process exits, whether or not this entry point is used.  The call allocates and frees nothing.
+ *
+ *   desc, x_dev, comp_dev, comp_capacity, seed, cuda_stream   exactly as for div_compress
+ *
+ * Returns what div_compress returns, and additionally
+ *   DIV_ERR_CAPACITY  when desc->n > DIV_STATIC_MAX_SAMPLES (the fixed scratch is too small; use div_compress),
+ *   DIV_ERR_CUDA      when the address of the array cannot be obtained on the current device.
+ *
+ * Things to know:
+ *   - the first call on each device looks up the device address of the array (a host-side runtime query
+ *     with that device current); make that first call outside any stream capture;
+ *   - all calls on one device share the one array.  Each call clears the part it uses before its kernel
+ *     runs (on the given stream), so earlier contents do not matter, but two calls whose work overlaps on
+ *     the GPU (different streams, or different host threads without ordering between their streams) race
+ *     on it and produce wrong output.  Keep calls on a device ordered one after the other;
+ *   - the output is byte-for-byte what div_compress writes for the same arguments;
+ *   - the device-side status word (see div_read_device_status) lives in the array and is not exposed.
+ */
+#define DIV_STATIC_MAX_SAMPLES 1024
+div_status div_compress_static(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                               uint64_t seed, void* cuda_stream);
+
+/*
  * Decompress (Sec. 4.2; Algorithm 1, backward loop): x_hat = UpSampling(H^L) + Delta*V^H + delta,
  * rounded to x_dtype.
  *   comp_dev    device; a blob written by div_compress with the SAME desc; read only

@@ -21,7 +21,7 @@ DIV_FLAG_NO_LAGGED_KERNEL = 4
 DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 
 EXPORTED_SYMBOLS = (
-    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_decompress", "div_plan_query",
+    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_decompress", "div_plan_query",
     "div_read_device_status", "div_status_string",
 )
 
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.div_compress.restype = c_int32
         L.div_compress_ex.argtypes = L.div_compress.argtypes + [c_uint32]
         L.div_compress_ex.restype = c_int32
+        L.div_compress_static.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_void_p, c_size_t, c_uint64, c_void_p]
+        L.div_compress_static.restype = c_int32
         L.div_decompress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_size_t, c_void_p, c_void_p]
         L.div_decompress.restype = c_int32
         L.div_plan_query.argtypes = [ctypes.POINTER(DivDesc), c_uint32, ctypes.POINTER(DivPlan)]
@@ -113,6 +115,20 @@ def div_compress(desc: DivDesc, x_ptr: int, comp_ptr: int, comp_capacity: int, w
                                c_void_p(ws_ptr), ws_bytes, c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream),
                                int(flags))
     _check(st, "div_compress")
+
+
+DIV_STATIC_MAX_SAMPLES = 1024
+
+
+def div_compress_static(desc: DivDesc, x_ptr: int, comp_ptr: int, comp_capacity: int, seed: int, stream: int = 0) -> None:
+    """div_compress with the scratch taken from a fixed array inside the library (nothing is allocated).
+
+    For callers that cannot allocate device memory where they compress; at most DIV_STATIC_MAX_SAMPLES
+    samples; calls on one device must not overlap on the GPU (they share the array).
+    """
+    st = lib().div_compress_static(ctypes.byref(desc), c_void_p(x_ptr), c_void_p(comp_ptr), comp_capacity,
+                                   c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream))
+    _check(st, "div_compress_static")
 
 
 def div_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xhat_ptr: int, stream: int = 0) -> None:

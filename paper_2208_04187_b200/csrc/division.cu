@@ -5,6 +5,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "decompress.cuh"
 #include "fused.cuh"
@@ -292,6 +294,61 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
             return launch_status();
         });
     });
+}
+
+// ------------------------------------------------------------------------------------------------
+// div_compress_static: compress with the scratch in a fixed array inside the library
+// ------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+// Scratch of div_compress_static: header + one 128-byte slot per sample, for up to
+// DIV_STATIC_MAX_SAMPLES samples.  It lives in every GPU that loads the library until the process ends.
+constexpr size_t STATIC_WS_BYTES =
+    (4ull * (divk::WS_HEADER_WORDS + (size_t)divk::WS_SLOT_WORDS * DIV_STATIC_MAX_SAMPLES) + 255ull) / 256ull * 256ull;
+static __device__ __align__(256) unsigned char g_static_workspace[STATIC_WS_BYTES];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[STATIC_MAX_DEVICES] = {};     // device address of the array, per device ordinal
+
+// Device address of g_static_workspace on the current device.  In host code the array's name is only a
+// handle for the runtime, not an address a kernel could use, so the address is asked for once per device.
+div_status static_workspace_ptr(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+        cudaGetLastError();
+        return DIV_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return DIV_ERR_CUDA;
+        }
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return DIV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+div_status div_compress_static(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                               uint64_t seed, void* cuda_stream) {
+    if (!desc) return DIV_ERR_NULL;
+    const div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (desc->n > DIV_STATIC_MAX_SAMPLES) return DIV_ERR_CAPACITY;      // the fixed scratch has no slot for more samples
+    void* ws = nullptr;
+    const div_status got = static_workspace_ptr(&ws);
+    if (got != DIV_OK) return got;
+    // same path as div_compress from here on (it clears the part of the scratch it uses on the stream)
+    return div_compress_ex(desc, x_dev, comp_dev, comp_capacity, ws, STATIC_WS_BYTES, seed, cuda_stream, 0u);
 }
 
 div_status div_read_device_status(const void* workspace_dev, void* cuda_stream, int32_t* out_status) {
