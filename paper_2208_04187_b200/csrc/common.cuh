@@ -131,6 +131,12 @@ __device__ __forceinline__ uint32_t quant4(float r0, float r1, float r2, float r
     return acc - BIAS;
 }
 
+// Dequantise one code (Sec. 4.2): fl(fl(Delta * code) + delta).
+__device__ __forceinline__ float dequantise(uint32_t code, float step, float delta) {
+    const float cf = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f);   // (float)code, exact
+    return __fadd_rn(__fmul_rn(step, cf), delta);
+}
+
 // Dequantise and reconstruct one element (Sec. 4.2): x_hat = lfc + (Delta * code + delta).
 __device__ __forceinline__ float reconstruct(uint32_t code, float step, float delta, float lfc) {
     const float cf = __fsub_rn(__uint_as_float(0x4B000000u | code), 8388608.0f);   // (float)code, exact

@@ -81,15 +81,72 @@ template <> struct Quad<__nv_bfloat16> {
     }
 };
 
+// Dequantisation through a table (Sec. 4.2: H^H_hat = Delta * V^H + delta).  A sample has only 2^Q
+// different values of fl(fl(Delta * code) + delta), so a CTA (which works inside one sample) builds them
+// once in shared memory, indexed by the packed bits of several codes at a time:
+//   Q = 1: 4 codes (a nibble)  -> 16 entries of 4 values      Q = 2: 4 codes (a byte) -> 256 entries of 4 values
+//   Q = 4: 2 codes (a byte)    -> 256 entries of 2 values     Q = 8: 1 code           -> 256 entries of 1 value
+template <int Q> struct DeqTable;
+template <> struct DeqTable<1> {
+    float4 t[16];
+    __device__ __forceinline__ void build(float step, float delta) {
+        if (threadIdx.x < 16) {
+            const uint32_t i = threadIdx.x;
+            t[i] = make_float4(dequantise(i & 1u, step, delta), dequantise((i >> 1) & 1u, step, delta),
+                               dequantise((i >> 2) & 1u, step, delta), dequantise((i >> 3) & 1u, step, delta));
+        }
+    }
+    __device__ __forceinline__ float4 quad(uint32_t bits) const { return t[bits & 15u]; }
+};
+template <> struct DeqTable<2> {
+    float4 t[256];
+    __device__ __forceinline__ void build(float step, float delta) {
+        const uint32_t i = threadIdx.x;
+        if (i < 256)
+            t[i] = make_float4(dequantise(i & 3u, step, delta), dequantise((i >> 2) & 3u, step, delta),
+                               dequantise((i >> 4) & 3u, step, delta), dequantise((i >> 6) & 3u, step, delta));
+    }
+    __device__ __forceinline__ float4 quad(uint32_t bits) const { return t[bits & 255u]; }
+};
+template <> struct DeqTable<4> {
+    float2 t[256];
+    __device__ __forceinline__ void build(float step, float delta) {
+        const uint32_t i = threadIdx.x;
+        if (i < 256) t[i] = make_float2(dequantise(i & 15u, step, delta), dequantise((i >> 4) & 15u, step, delta));
+    }
+    __device__ __forceinline__ float4 quad(uint32_t bits) const {
+        const float2 a = t[bits & 255u], b = t[(bits >> 8) & 255u];
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+};
+template <> struct DeqTable<8> {
+    float t[256];
+    __device__ __forceinline__ void build(float step, float delta) {
+        const uint32_t i = threadIdx.x;
+        if (i < 256) t[i] = dequantise(i, step, delta);
+    }
+    __device__ __forceinline__ float4 quad(uint32_t bits) const {
+        return make_float4(t[bits & 255u], t[(bits >> 8) & 255u], t[(bits >> 16) & 255u], t[bits >> 24]);
+    }
+};
+
+// the packed bits of quad number `quad` (global numbering) of the code stream
+template <int Q>
+__device__ __forceinline__ uint32_t quad_bits(const uint32_t* __restrict__ packed, uint64_t quad) {
+    if (Q == 2) return __ldg(reinterpret_cast<const uint8_t*>(packed) + quad);
+    if (Q == 4) return __ldg(reinterpret_cast<const uint16_t*>(packed) + quad);
+    if (Q == 8) return __ldg(packed + quad);
+    return (__ldg(reinterpret_cast<const uint8_t*>(packed) + (quad >> 1)) >> (4u * (uint32_t)(quad & 1u))) & 15u;
+}
+
 template <typename XT, typename LT, int Q, int QPT>
 __global__ void __launch_bounds__(256)
 decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
-    constexpr uint32_t QMASK = (1u << Q) - 1u;
-    constexpr uint32_t GMASK = (Q == 8) ? 0xFFFFFFFFu : ((1u << (4 * Q)) - 1u);
+    __shared__ DeqTable<Q> table;
     const uint32_t n = blockIdx.y;
-    const float delta = __ldg(stats + 2 * (size_t)n);
-    const float step = __ldg(stats + 2 * (size_t)n + 1);
+    table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
+    __syncthreads();
     const uint64_t sample_quad0 = (uint64_t)n * d.qps;
     const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
     const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
@@ -100,8 +157,7 @@ decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
     for (int k = 0; k < QPT; ++k) {
         const uint32_t q = q0 + k * 256u;
         if (q < d.qps) {
-            const uint64_t bitpos = (sample_quad0 + q) * (4u * Q);
-            bits[k] = (__ldg(packed + (bitpos >> 5)) >> (uint32_t)(bitpos & 31u)) & GMASK;
+            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
             const uint32_t plane = fdiv(q, d.by_hwq);
             const uint32_t rem = q - plane * d.hwq;
             const uint32_t h = fdiv(rem, d.by_wq);
@@ -113,12 +169,63 @@ decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
     for (int k = 0; k < QPT; ++k) {
         const uint32_t q = q0 + k * 256u;
         if (q < d.qps) {
-            const uint32_t b = bits[k];
-            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u,
-                            reconstruct(b & QMASK, step, delta, lf[k]),
-                            reconstruct((b >> Q) & QMASK, step, delta, lf[k]),
-                            reconstruct((b >> (2 * Q)) & QMASK, step, delta, lf[k]),
-                            reconstruct((b >> (3 * Q)) & QMASK, step, delta, lf[k]));
+            const float4 hq = table.quad(bits[k]);
+            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, __fadd_rn(lf[k], hq.x), __fadd_rn(lf[k], hq.y),
+                            __fadd_rn(lf[k], hq.z), __fadd_rn(lf[k], hq.w));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// flat kernel: any W and B, sample size a multiple of 4 elements, planes of at most FLAT_MAX_HW
+// elements.  One thread produces QPT quads of 4 consecutive elements (global flat order), which may
+// lie in different tiles, rows or planes: the tile of every position of a plane comes from a table
+// in shared memory (built once per CTA), the plane index advances with the position.
+// grid = (ceil(quads_per_sample / (256*QPT)), N), dynamic shared memory = 2 * HW bytes
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t FLAT_MAX_HW = 8192;
+
+struct DecFlat {
+    uint32_t qps;        // quads per sample = CHW / 4
+    uint32_t C, TPP, Wb, HW, W, B;
+    FastDiv by_hw, by_w, by_b;
+};
+
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                       const float* __restrict__ stats, XT* __restrict__ xhat, DecFlat d) {
+    extern __shared__ uint16_t tile_of[];      // position inside a plane -> tile inside the plane
+    __shared__ DeqTable<Q> table;
+    const uint32_t n = blockIdx.y;
+    table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
+    for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
+        const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
+        tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
+    }
+    __syncthreads();
+    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
+    const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < d.qps) {
+            const float4 hq = table.quad(quad_bits<Q>(packed, sample_quad0 + q));
+            const float hv[4] = {hq.x, hq.y, hq.z, hq.w};
+            uint32_t plane = fdiv(q * 4u, d.by_hw);
+            uint32_t rem = q * 4u - plane * d.HW;
+            const LT* lfc_p = lfc_n + (size_t)plane * d.TPP;
+            float v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                v[i] = __fadd_rn(Elem<LT>::load(lfc_p + tile_of[rem]), hv[i]);
+                if (++rem == d.HW) {
+                    rem = 0;
+                    lfc_p += d.TPP;
+                }
+            }
+            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, v[0], v[1], v[2], v[3]);
         }
     }
 }

@@ -141,6 +141,9 @@ constexpr int DEC_QPT = 4;
 bool decompress_fast_ok(const Shape& s) {
     return (s.W % 4 == 0) && s.B >= 4 && (s.B & (s.B - 1)) == 0 && s.N <= 65535;
 }
+bool decompress_flat_ok(const Shape& s) {
+    return (s.CHW % 4 == 0) && s.HW <= FLAT_MAX_HW && s.TPP <= 65535 && s.N <= 65535 && s.CHW < (1u << 31);
+}
 
 }  // namespace
 
@@ -210,7 +213,7 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
         out->grid = (int32_t)((s.tiles + 255) / 256);
         out->threads = 256;
     }
-    out->decompress_fast = decompress_fast_ok(s) ? 1 : 0;
+    out->decompress_fast = decompress_fast_ok(s) ? 1 : (decompress_flat_ok(s) ? 2 : 0);
     return DIV_OK;
 }
 
@@ -286,6 +289,21 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 const uint32_t per_block = 256u * DEC_QPT;
                 dim3 grid((d.qps + per_block - 1) / per_block, s.N);
                 decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+            } else if (decompress_flat_ok(s)) {
+                DecFlat d;
+                d.qps = s.CHW / 4;
+                d.C = s.C;
+                d.TPP = s.TPP;
+                d.Wb = s.Wb;
+                d.HW = s.HW;
+                d.W = s.W;
+                d.B = s.B;
+                d.by_hw = make_fastdiv(s.HW);
+                d.by_w = make_fastdiv(s.W);
+                d.by_b = make_fastdiv(s.B);
+                const uint32_t per_block = 256u * DEC_QPT;
+                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 2u * s.HW, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
             } else {
                 const uint64_t g = (nwords + 255) / 256;
                 if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
