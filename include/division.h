@@ -93,6 +93,8 @@ typedef struct div_plan {
                                   (W%4==0, B in {4,8}, Q in {2,4,8});
                                3: one launch, x read from HBM once and re-read from L2 a little later
                                   (same shapes; taken when the ring cannot hold a sample's share);
+                               4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
+                                  at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
@@ -111,6 +113,7 @@ typedef struct div_plan {
 #define DIV_FLAG_FORCE_TWO_PASS 1u   /* never take a fused kernel                          */
 #define DIV_FLAG_NO_STRIP_KERNEL 2u  /* never take the strip variant of the ring kernel    */
 #define DIV_FLAG_NO_LAGGED_KERNEL 4u /* never take the lagged (L2 re-read) kernel          */
+#define DIV_FLAG_NO_PLANE_KERNELS 8u /* never take the small-plane pair of kernels          */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:

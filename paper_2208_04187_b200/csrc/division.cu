@@ -12,6 +12,7 @@
 #include "fused.cuh"
 #include "fused_v.cuh"
 #include "lagged.cuh"
+#include "planes.cuh"
 #include "twopass.cuh"
 
 namespace {
@@ -20,7 +21,8 @@ using namespace divk;
 typedef __nv_bfloat16 bf16;
 
 constexpr uint64_t SECTION_ALIGN = 128;
-constexpr uint32_t DIV_FLAG_ALL = DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL;
+constexpr uint32_t DIV_FLAG_ALL =
+    DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL | DIV_FLAG_NO_PLANE_KERNELS;
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
@@ -183,8 +185,10 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     LPlan lp;
     const bool vec = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
     const bool lag = !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
-    const bool fused = !lag && !vec && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
-    out->fused = lag ? 3 : (vec ? 2 : (fused ? 1 : 0));
+    PlaneGeom pg;
+    const bool planes = !lag && !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS)) && plan_planes(desc, s, &pg);
+    const bool fused = !lag && !vec && !planes && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
+    out->fused = lag ? 3 : (vec ? 2 : (planes ? 4 : (fused ? 1 : 0)));
     if (lag) {
         out->grid = lp.grid;
         out->threads = lp.threads;
@@ -201,6 +205,10 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
         out->smem_bytes = vp.smem_bytes;
         out->chunk_elems = vp.chunk_elems;
         out->chunks_per_sample = vp.chunks_per_sample;
+    } else if (planes) {
+        out->grid = (int32_t)((pg.qps + 256 * PLANE_QPT - 1) / (256 * PLANE_QPT) * s.N);
+        out->threads = 256;
+        out->chunk_elems = 4 * PLANE_QPT * 256;
     } else if (fused) {
         out->grid = fp.grid;
         out->threads = fp.threads;
@@ -233,6 +241,10 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
     uint8_t* blob = (uint8_t*)comp_dev;
     uint32_t* ws = (uint32_t*)workspace_dev;
+    // kernels that store bytes or half-words leave the unused top of a partial last word alone: it is zero by contract
+    if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
+        cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
+        return DIV_ERR_CUDA;
     if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL))) {
         VPlan vp;
         if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream);
@@ -240,6 +252,10 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL))) {
         LPlan lp;
         if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
+    }
+    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS))) {
+        PlaneGeom pg;
+        if (plan_planes(desc, s, &pg)) return compress_planes(desc, s, lo, pg, x_dev, blob, ws, seed, stream);
     }
     if (!(flags & DIV_FLAG_FORCE_TWO_PASS)) {
         FusedPlan fp;

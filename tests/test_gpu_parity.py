@@ -17,7 +17,8 @@ pytestmark = pytest.mark.gpu
 
 TWO_PASS = binding.DIV_FLAG_FORCE_TWO_PASS
 LAGGED = binding.DIV_FLAG_NO_STRIP_KERNEL          # skip the strip ring kernel: the lagged kernel is next in line
-NO_STRIP = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL
+NO_STRIP = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL | binding.DIV_FLAG_NO_PLANE_KERNELS
+NO_SPECIAL = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL      # planes pair, else general ring
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -109,6 +110,14 @@ SMALL = [
     (3, 20, 24, 40, 4, 2, "f32", "f32"),
     (2, 9, 36, 20, 8, 2, "f32", "f32"),
     (5, 11, 12, 52, 8, 2, "bf16", "bf16"),
+    # small planes of odd width: the pair of plane kernels
+    (3, 12, 14, 14, 8, 2, "f32", "f32"),
+    (2, 20, 7, 7, 8, 2, "f32", "bf16"),
+    (2, 8, 14, 14, 8, 4, "bf16", "bf16"),
+    (2, 4, 13, 9, 4, 2, "f32", "f32"),
+    (3, 4, 21, 27, 16, 8, "f32", "f32"),
+    (2, 8, 7, 7, 4, 2, "bf16", "f32"),
+    (1, 4, 30, 10, 8, 2, "f32", "f32"),
 ]
 
 
@@ -118,36 +127,52 @@ def small_input(n, c, h, w, x_dtype, seed):
 
 
 @pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(map(str, c)))
-@pytest.mark.parametrize("flags", [0, LAGGED, NO_STRIP, TWO_PASS], ids=["default", "lagged", "general_ring", "two_pass"])
+@pytest.mark.parametrize("flags", [0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS], ids=["default", "lagged", "planes", "general_ring", "two_pass"])
 def test_small_cases_match_the_checker(case, flags):
     n, c, h, w, block, q, xd, ld = case
     x = small_input(n, c, h, w, xd, seed=n + c + h + w + block + q)
     assert_full_parity(x, block, q, seed=1234567, x_dtype=xd, lfc_dtype=ld, flags=flags)
 
 
+def planes_shape(case):
+    n, c, h, w, block, q, xd, ld = case
+    b = min(block, max(h, w))
+    p2 = 1
+    while p2 < b:
+        p2 *= 2
+    wb = -(-w // b)
+    return q in (2, 4, 8) and p2 in (4, 8, 16) and wb * p2 <= 32 and (c * h * w) % 4 == 0 and h * w <= 8192
+
+
 def test_fused_path_is_taken_where_expected():
     """Guards against silently testing only the general kernels."""
     fused = {case: binding.div_plan_query(binding.make_desc(*case)).fused for case in SMALL}
     lagged = {case: binding.div_plan_query(binding.make_desc(*case), LAGGED).fused for case in SMALL}
+    special = {case: binding.div_plan_query(binding.make_desc(*case), NO_SPECIAL).fused for case in SMALL}
     for case in SMALL:
         n, c, h, w, block, q, xd, ld = case
         strip_shape = w % 4 == 0 and min(block, max(h, w)) in (4, 8) and q in (2, 4, 8)
         if strip_shape:
             assert fused[case] == 2 and lagged[case] == 3, case
+        elif planes_shape(case):
+            assert fused[case] == 4 and lagged[case] == 4, case
         else:
             assert fused[case] in (0, 1) and lagged[case] == fused[case], case
+        assert special[case] == (4 if planes_shape(case) else binding.div_plan_query(binding.make_desc(*case), NO_STRIP).fused), case
     assert sum(1 for c in SMALL if fused[c] == 2) >= 12
+    assert sum(1 for c in SMALL if fused[c] == 4) >= 5
+    assert sum(1 for c in SMALL if special[c] == 4) >= 12
     assert fused[(2, 4, 32, 32, 8, 1, "f32", "f32")] == 1          # Q = 1: general ring kernel
-    assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 1
-    assert fused[(2, 16, 7, 7, 8, 2, "f32", "f32")] == 1
-    assert fused[(2, 3, 40, 24, 16, 2, "f32", "f32")] == 1
+    assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 4
+    assert fused[(2, 16, 7, 7, 8, 2, "f32", "f32")] == 4
+    assert fused[(2, 3, 40, 24, 16, 2, "f32", "f32")] == 4
     assert binding.div_plan_query(binding.make_desc(3, 4, 32, 32, 8, 2), NO_STRIP).fused == 1
     assert fused[(1, 2, 3, 3, 2, 2, "f32", "f32")] == 0          # sample is not a whole number of words
     assert fused[(2, 2, 70, 70, 64, 2, "f32", "f32")] == 0        # block wider than a warp
     for spec in synth.config2() + synth.config1() + synth.config3():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
-        assert binding.div_plan_query(d).fused == (2 if spec.w % 4 == 0 else 1), spec.label()
-        assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 1), spec.label()
+        assert binding.div_plan_query(d).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
+        assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d).decompress_fast == (1 if spec.w % 4 == 0 else 2)
 
 
@@ -204,7 +229,7 @@ def test_guard_bands_stay_untouched():
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
                  (2, 8, 32, 32, 8, 2, "bf16", "bf16")]:
         n, c, h, w, block, q, xd, ld = case
-        for flags in (0, LAGGED, NO_STRIP, TWO_PASS):
+        for flags in (0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
             x = small_input(n, c, h, w, xd, seed=7)
             codec = binding.Codec(n, c, h, w, block, q, xd, ld)
             pad = 4096
@@ -257,7 +282,7 @@ def assert_sampled_parity(spec, seed, sample_ids, flags=0):
 def test_config0_full():
     spec = synth.config0()[0]
     x = synth.make_input(spec)
-    for flags in (0, LAGGED, NO_STRIP, TWO_PASS):
+    for flags in (0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
         assert_full_parity(x, spec.block, spec.qbits, 0, flags=flags)
 
 
