@@ -189,6 +189,18 @@ div_status div_compress_static(const div_desc* desc, const void* x_dev, void* co
 div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes,
                           void* xhat_dev, void* cuda_stream);
 
+/*
+ * Test hook for the bounded waits of the single-launch compress kernels (plan codes 2 and 3): runs the
+ * kernel div_compress_ex would run, but tells it to wait for a number of arrivals per sample that is never
+ * reached, with `timeout_ns` (at most 100 ms) as the limit of every wait.  The kernel must give up, record
+ * DIV_ERR_TIMEOUT in the workspace status word (read it with div_read_device_status) and return; the blob's
+ * contents are then unspecified.  Returns DIV_ERR_PARAM when the descriptor maps to neither kernel.
+ * Arguments as for div_compress_ex.  No counterpart in the paper.
+ */
+div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                                      void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream,
+                                      uint32_t flags, uint64_t timeout_ns);
+
 /* Which kernels a descriptor maps to on the current device.  desc, out: host. */
 div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
 

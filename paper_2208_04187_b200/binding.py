@@ -22,7 +22,8 @@ DIV_FLAG_NO_PLANE_KERNELS = 8
 DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 
 EXPORTED_SYMBOLS = (
-    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_decompress", "div_plan_query",
+    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_debug_compress_starved",
+    "div_decompress", "div_plan_query",
     "div_read_device_status", "div_status_string",
 )
 
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.div_compress_ex.restype = c_int32
         L.div_compress_static.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_void_p, c_size_t, c_uint64, c_void_p]
         L.div_compress_static.restype = c_int32
+        L.div_debug_compress_starved.argtypes = L.div_compress_ex.argtypes + [c_uint64]
+        L.div_debug_compress_starved.restype = c_int32
         L.div_decompress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_size_t, c_void_p, c_void_p]
         L.div_decompress.restype = c_int32
         L.div_plan_query.argtypes = [ctypes.POINTER(DivDesc), c_uint32, ctypes.POINTER(DivPlan)]

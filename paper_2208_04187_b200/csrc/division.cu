@@ -264,6 +264,34 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
 }
 
+div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                                      void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream,
+                                      uint32_t flags, uint64_t timeout_ns) {
+    if (!desc || !x_dev || !comp_dev || !workspace_dev) return DIV_ERR_NULL;
+    div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if ((flags & ~DIV_FLAG_ALL) || timeout_ns == 0 || timeout_ns > 100000000ull) return DIV_ERR_PARAM;
+    if (!aligned16(x_dev) || !aligned16(comp_dev) || !aligned16(workspace_dev)) return DIV_ERR_ALIGN;
+    const Shape s = make_shape(desc);
+    div_layout lo;
+    make_layout(desc, s, &lo);
+    if (comp_capacity < lo.total_bytes || workspace_bytes < lo.workspace_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
+    uint8_t* blob = (uint8_t*)comp_dev;
+    uint32_t* ws = (uint32_t*)workspace_dev;
+    const uint32_t never = 0xFFFFFFFFu;      // an arrival count no sample reaches
+    if (!(flags & DIV_FLAG_NO_STRIP_KERNEL)) {
+        VPlan vp;
+        if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream, never, timeout_ns);
+    }
+    if (!(flags & DIV_FLAG_NO_LAGGED_KERNEL)) {
+        LPlan lp;
+        if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream, never, timeout_ns);
+    }
+    return DIV_ERR_PARAM;
+}
+
 div_status div_compress(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
                         void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream) {
     return div_compress_ex(desc, x_dev, comp_dev, comp_capacity, workspace_dev, workspace_bytes, seed, cuda_stream, 0u);

@@ -224,6 +224,31 @@ def test_same_seed_same_bytes_other_seed_other_codes():
     assert (wa != wc).mean() > 0.5
 
 
+@pytest.mark.parametrize("flags", [0, LAGGED], ids=["strip_ring", "lagged"])
+def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
+    """Failure detection without a fault: the kernel waits for arrivals that never come, its 2 ms limit
+    runs out, it records the timeout in the status word and returns; the context stays usable."""
+    import ctypes
+    spec = synth.config0()[0]
+    x = to_device(synth.make_input(spec), "f32")
+    codec = binding.Codec(*spec.shape, spec.block, spec.qbits)
+    assert codec.plan(flags).fused == (3 if flags else 2)
+    st = binding.lib().div_debug_compress_starved(
+        ctypes.byref(codec.desc), ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(codec.blob.data_ptr()), codec.blob.numel(),
+        ctypes.c_void_p(codec.workspace.data_ptr()), codec.workspace.numel(), 0, ctypes.c_void_p(binding.current_stream_handle()),
+        flags, 2_000_000)
+    assert st == binding.DIV_OK
+    torch.cuda.synchronize()
+    assert codec.device_status() == binding.DIV_ERR_TIMEOUT
+    # the next ordinary call on the same buffers works and is correct
+    ref = orc.compress(synth.make_input(spec), spec.block, spec.qbits, 5)
+    codec.compress(x, seed=5, flags=flags)
+    torch.cuda.synchronize()
+    assert codec.device_status() == binding.DIV_OK
+    _, words, _ = split_blob(codec.blob.cpu().numpy(), codec.layout, "f32")
+    np.testing.assert_array_equal(words, ref.words)
+
+
 def test_guard_bands_stay_untouched():
     """Sentinel bytes around every output buffer survive both calls (no out-of-bounds write)."""
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
