@@ -89,10 +89,10 @@ typedef struct div_layout {
 
 /* How div_compress will run a descriptor (introspection for tests and benchmarks). */
 typedef struct div_plan {
-    int32_t fused;          /* 2: one launch, chunks wait in a shared-memory ring, strip kernel
-                                  (W%4==0, B in {4,8}, Q in {2,4,8});
-                               3: one launch, x read from HBM once and re-read from L2 a little later
-                                  (same shapes; taken when the ring cannot hold a sample's share);
+    int32_t fused;          /* for W%4==0, B in {4,8}, Q in {2,4,8}, one launch:
+                               2: chunks wait in a shared-memory ring (strip ring kernel; first choice below 40 MB);
+                               3: x read from HBM once and re-read from L2 a little later (lagged kernel; first
+                                  choice from 40 MB up, and whenever the ring cannot hold a sample's share);
                                4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
                                   at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels */

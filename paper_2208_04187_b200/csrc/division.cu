@@ -140,6 +140,12 @@ div_status compress_two_pass(const div_desc* d, const Shape& s, const div_layout
 // ------------------------------------------------------------------------------------------
 constexpr int DEC_QPT = 4;
 
+// Large maps go to the lagged kernel first (measured: a few per cent faster from about 40 MB up), small ones
+// to the strip ring kernel (shorter start-up).
+bool prefer_lagged(const div_desc* d, const Shape& s) {
+    return s.total * dtype_bytes(d->x_dtype) >= (40ull << 20);
+}
+
 bool decompress_fast_ok(const Shape& s) {
     return (s.W % 4 == 0) && s.B >= 4 && (s.B & (s.B - 1)) == 0 && s.N <= 65535;
 }
@@ -183,8 +189,11 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     FusedPlan fp;
     VPlan vp;
     LPlan lp;
-    const bool vec = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
-    const bool lag = !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
+    const bool lag_first = prefer_lagged(desc, s);
+    const bool lag_ok = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
+    const bool vec_ok = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
+    const bool lag = lag_ok && (lag_first || !vec_ok);
+    const bool vec = vec_ok && !lag;
     PlaneGeom pg;
     const bool planes = !lag && !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS)) && plan_planes(desc, s, &pg);
     const bool fused = !lag && !vec && !planes && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
@@ -245,14 +254,16 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
         cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
         return DIV_ERR_CUDA;
-    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL))) {
+    const bool may_lag = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL));
+    const bool may_strip = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL));
+    LPlan lp;
+    if (may_lag && prefer_lagged(desc, s) && plan_lagged(desc, s, &lp) == DIV_OK)
+        return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
+    if (may_strip) {
         VPlan vp;
         if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream);
     }
-    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL))) {
-        LPlan lp;
-        if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
-    }
+    if (may_lag && plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
     if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS))) {
         PlaneGeom pg;
         if (plan_planes(desc, s, &pg)) return compress_planes(desc, s, lo, pg, x_dev, blob, ws, seed, stream);

@@ -15,7 +15,7 @@
 //     set-up arithmetic of a lane is paid once per J bands, and from one band to the next every index
 //     advances by a constant.
 //   * warps are independent: each claims the next unit from a counter in global scratch (one atomic
-//     per unit, issued one unit ahead), reduces it, folds its residual extremes into the sample's slot
+//     per unit), reduces it at once, folds its residual extremes into the sample's slot
 //     in global scratch and counts the unit as arrived; the arrival that completes a sample derives
 //     (delta, Delta, scale), writes the first two to the blob and publishes all of it in the slot.
 //   * the quantise half reads the slot (bounded wait; normally the first look succeeds), re-reads the
@@ -37,10 +37,10 @@ namespace divk {
 #define DIVK_L_WARPS 8
 #endif
 #ifndef DIVK_L_MIN_CTAS
-#define DIVK_L_MIN_CTAS 4
+#define DIVK_L_MIN_CTAS 2
 #endif
 #ifndef DIVK_L_LAG_BYTES
-#define DIVK_L_LAG_BYTES (24u << 20)
+#define DIVK_L_LAG_BYTES (16u << 20)
 #endif
 #ifndef DIVK_L_BANDS
 #define DIVK_L_BANDS 4
@@ -93,6 +93,11 @@ __device__ __forceinline__ uint64_t l2_policy_release() {
     asm("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
+__device__ __forceinline__ uint32_t atom_add_release(uint32_t* p, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.release.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 // a strip row from global memory as two packed pairs (x, y) and (z, w), widened to fp32
 template <typename XT> struct GlobalRow2;
 template <> struct GlobalRow2<float> {
@@ -138,6 +143,74 @@ __device__ __forceinline__ LStart l_start(const LParams& p, uint32_t uu, uint32_
     return t;
 }
 
+// the B rows of one full band of a strip
+template <typename XT, int P2>
+__device__ __forceinline__ void l_load_band(const unsigned char* xs, uint32_t row_bytes, uint64_t pol,
+                                            uint64_t (&vxy)[P2], uint64_t (&vzw)[P2]) {
+#pragma unroll
+    for (int r = 0; r < P2; ++r) GlobalRow2<XT>::load(xs + r * row_bytes, pol, vxy[r], vzw[r]);
+}
+
+// reduce half of one full band (all B rows in bounds): tile mean in the fixed order, stored low-frequency
+// value, extremes of the residual folded into (lo, hi)
+template <typename LT, int P2>
+__device__ __forceinline__ void l_reduce_full_band(const uint64_t (&vxy)[P2], const uint64_t (&vzw)[P2], float inv,
+                                                   float cnt, bool writer, bool live, LT* lfc_n, float& lo, float& hi) {
+    constexpr uint32_t LPT = P2 / 4;
+    uint64_t cxy[P2], czw[P2];
+#pragma unroll
+    for (int r = 0; r < P2; ++r) {
+        cxy[r] = vxy[r];
+        czw[r] = vzw[r];
+    }
+#pragma unroll
+    for (int w = P2; w > 1; w >>= 1) {
+#pragma unroll
+        for (int i = 0; i < w / 2; ++i) {
+            cxy[i] = add2_rn(cxy[2 * i], cxy[2 * i + 1]);
+            czw[i] = add2_rn(czw[2 * i], czw[2 * i + 1]);
+        }
+    }
+    float c0, c1, c2, c3;
+    upk2(cxy[0], c0, c1);
+    upk2(czw[0], c2, c3);
+    float sum = __fadd_rn(__fadd_rn(c0, c1), __fadd_rn(c2, c3));
+#pragma unroll
+    for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+    const float mean = (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, cnt);
+    const float stored = Elem<LT>::round(mean);
+    if (live) {
+        if (writer) Elem<LT>::store(lfc_n, mean);
+        float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+#pragma unroll
+        for (int r = 0; r < P2; ++r) {
+            float a_, b_, c_, d_;
+            upk2(vxy[r], a_, b_);
+            upk2(vzw[r], c_, d_);
+            blo = fmin3(blo, a_, b_);
+            blo = fmin3(blo, c_, d_);
+            bhi = fmax3(bhi, a_, b_);
+            bhi = fmax3(bhi, c_, d_);
+        }
+        lo = fminf(lo, __fsub_rn(blo, stored));
+        hi = fmaxf(hi, __fsub_rn(bhi, stored));
+    }
+}
+
+// quantise half of one full band: B rows of 4 codes each
+template <typename OutT, int Q, int P2>
+__device__ __forceinline__ void l_quant_full_band(const uint64_t (&vxy)[P2], const uint64_t (&vzw)[P2], float stored,
+                                                  uint64_t delta2, uint64_t scale2, uint64_t& ctr, uint64_t row_step,
+                                                  OutT*& out, uint32_t W4) {
+    const uint64_t stored2 = pk2(stored, stored);
+#pragma unroll
+    for (int r = 0; r < P2; ++r) {
+        *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
+        out += W4;
+        ctr += row_step;
+    }
+}
+
 template <typename XT, typename LT, int Q, int P2>
 __global__ void __launch_bounds__(L_THREADS, DIVK_L_MIN_CTAS)
 lagged_kernel(const LParams p) {
@@ -165,7 +238,6 @@ lagged_kernel(const LParams p) {
     while (true) {
         const uint32_t j = __shfl_sync(0xFFFFFFFFu, next, 0);
         if (j >= TU + D) break;
-        if (lane == 0) next = atomicAdd(claim_word, 1u);        // the claim for the next turn travels meanwhile
 
         // ================= reduce half: unit j =================
         if (j < TU) {
@@ -178,6 +250,21 @@ lagged_kernel(const LParams p) {
             const bool all_full = __all_sync(0xFFFFFFFFu, t.nb == J) && (p.tail_rows == s.B);
             uint32_t bh = t.bh;
             float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+            if (all_full && J == 4u) {
+                // four full bands for every lane: two register buffers, the loads of a band are issued
+                // before the band in the other buffer is worked on
+                const uint32_t band_bytes = s.B * row_bytes;
+                const float inv = p.inv_cnt[tail_col], cnt = p.cnt[tail_col];
+                uint64_t axy[P2], azw[P2], bxy[P2], bzw[P2];
+                l_load_band<XT, P2>(xs, row_bytes, pol_keep, axy, azw);
+                l_load_band<XT, P2>(xs + band_bytes, row_bytes, pol_keep, bxy, bzw);
+                l_reduce_full_band<LT, P2>(axy, azw, inv, cnt, writer, true, lfc_n, lo, hi);
+                l_load_band<XT, P2>(xs + 2u * band_bytes, row_bytes, pol_keep, axy, azw);
+                l_reduce_full_band<LT, P2>(bxy, bzw, inv, cnt, writer, true, lfc_n + s.Wb, lo, hi);
+                l_load_band<XT, P2>(xs + 3u * band_bytes, row_bytes, pol_keep, bxy, bzw);
+                l_reduce_full_band<LT, P2>(axy, azw, inv, cnt, writer, true, lfc_n + 2u * s.Wb, lo, hi);
+                l_reduce_full_band<LT, P2>(bxy, bzw, inv, cnt, writer, true, lfc_n + 3u * s.Wb, lo, hi);
+            } else
             for (uint32_t jb = 0; jb < J; ++jb) {
                 const uint32_t rows = (jb < t.nb) ? ((bh + 1u == s.Hb) ? p.tail_rows : s.B) : 0u;
                 uint64_t vxy[P2], vzw[P2];
@@ -249,9 +336,10 @@ lagged_kernel(const LParams p) {
                 uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
                 red_max_relaxed(slot + 0, kmin);
                 red_max_relaxed(slot + 1, kmax);
-                const uint32_t before = atom_add_acq_rel(slot + 2, 1u);
+                const uint32_t before = atom_add_release(slot + 2, 1u);
                 if (before + 1u == p.expected_units) {
                     // this arrival completes the sample
+                    fence_acq_rel_gpu();
                     const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
                     p.stats[2 * (size_t)n + 0] = qp.delta;
                     p.stats[2 * (size_t)n + 1] = qp.step;
@@ -308,6 +396,20 @@ lagged_kernel(const LParams p) {
                     uint64_t ctr = rng_sample_base(p.seed, n) + K_GROUP * (uint64_t)(g0 + 1u);
                     OutT* out = packed + (((uint64_t)n * s.CHW) >> 2) + g0;
                     uint32_t bh = t.bh;
+                    if (t.nb == 4u && p.tail_rows == s.B) {
+                        const uint32_t band_bytes = s.B * row_bytes;
+                        const float st0 = Elem<LT>::load_cg(lfc_n), st1 = Elem<LT>::load_cg(lfc_n + s.Wb);
+                        const float st2 = Elem<LT>::load_cg(lfc_n + 2u * s.Wb), st3 = Elem<LT>::load_cg(lfc_n + 3u * s.Wb);
+                        uint64_t axy[P2], azw[P2], bxy[P2], bzw[P2];
+                        l_load_band<XT, P2>(xs, row_bytes, pol_release, axy, azw);
+                        l_load_band<XT, P2>(xs + band_bytes, row_bytes, pol_release, bxy, bzw);
+                        l_quant_full_band<OutT, Q, P2>(axy, azw, st0, delta2, scale2, ctr, p.rng_row_step, out, W4);
+                        l_load_band<XT, P2>(xs + 2u * band_bytes, row_bytes, pol_release, axy, azw);
+                        l_quant_full_band<OutT, Q, P2>(bxy, bzw, st1, delta2, scale2, ctr, p.rng_row_step, out, W4);
+                        l_load_band<XT, P2>(xs + 3u * band_bytes, row_bytes, pol_release, bxy, bzw);
+                        l_quant_full_band<OutT, Q, P2>(axy, azw, st2, delta2, scale2, ctr, p.rng_row_step, out, W4);
+                        l_quant_full_band<OutT, Q, P2>(bxy, bzw, st3, delta2, scale2, ctr, p.rng_row_step, out, W4);
+                    } else
                     for (uint32_t jb = 0; jb < t.nb; ++jb) {
                         const uint32_t rows = (bh + 1u == s.Hb) ? p.tail_rows : s.B;
                         const float stored = Elem<LT>::load_cg(lfc_n);
@@ -341,6 +443,9 @@ lagged_kernel(const LParams p) {
                 }
             }
         }
+        // claim the next unit only now: a claimed unit that waits behind this warp's quantise half would
+        // hold back its whole sample
+        if (lane == 0) next = atomicAdd(claim_word, 1u);
     }
 }
 

@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 
 TWO_PASS = binding.DIV_FLAG_FORCE_TWO_PASS
 LAGGED = binding.DIV_FLAG_NO_STRIP_KERNEL          # skip the strip ring kernel: the lagged kernel is next in line
+RING = binding.DIV_FLAG_NO_LAGGED_KERNEL           # skip the lagged kernel: the strip ring kernel where it applies
 NO_STRIP = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL | binding.DIV_FLAG_NO_PLANE_KERNELS
 NO_SPECIAL = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL      # planes pair, else general ring
 
@@ -171,8 +172,10 @@ def test_fused_path_is_taken_where_expected():
     assert fused[(2, 2, 70, 70, 64, 2, "f32", "f32")] == 0        # block wider than a warp
     for spec in synth.config2() + synth.config1() + synth.config3():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
-        assert binding.div_plan_query(d).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
+        big = spec.numel * (4 if spec.x_dtype == "f32" else 2) >= 40 * 2 ** 20
+        assert binding.div_plan_query(d).fused == ((3 if big else 2) if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 4), spec.label()
+        assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d).decompress_fast == (1 if spec.w % 4 == 0 else 2)
 
 
@@ -326,6 +329,8 @@ def test_config2_other_paths_on_one_tensor():
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=TWO_PASS)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=NO_STRIP)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=LAGGED)
+    assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=RING)
+    assert_sampled_parity(synth.config2()[0], 0, [17], flags=RING)
 
 
 @pytest.mark.parametrize("spec", synth.config3(), ids=lambda s: s.label())
