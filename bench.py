@@ -31,10 +31,10 @@ WORKLOAD = "config2: ResNet-50 ImageNet-shaped set, batch 64 fp32, B=8, Q=2, fp3
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes per launch of the dominant kernel (strip ring compress kernel on the 64x64x112x112 map):
+# DRAM bytes per launch of the dominant kernel (lagged compress kernel on the 64x64x112x112 map):
 # dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture, see profiles/.  Set to None whenever that
 # kernel changes after the capture.
-NCU_TRAFFIC_BYTES = 217896960      # 205566464 read + 12330496 written (profiles/fused_v_and_decompress_quad_map_64x64x112x112.md)
+NCU_TRAFFIC_BYTES = 214477824      # 206767872 read + 7709952 written (profiles/lagged_kernel_and_decompress_quad_map_64x64x112x112.md)
 
 
 def measured_peak():
@@ -201,7 +201,7 @@ def run_ours(args):
     dev_x = [h.to(device, non_blocking=True) for h in host_x]
     codecs = [binding.Codec(*s.shape, s.block, s.qbits, s.x_dtype, s.lfc_dtype, device=device) for s in specs]
     dev_out = [torch.empty_like(x) for x in dev_x]
-    plans = [c.plan() for c in codecs]
+    plans = [c.plan(args.compress_flags) for c in codecs]
     raw_bytes = sum(int(c.layout.raw_bytes) for c in codecs)
     comp_bytes = sum(int(c.layout.closed_form_bytes) for c in codecs)
     kernels_per_step = sum((2 if p.fused in (0, 4) else 1) + 1 for p in plans)
@@ -211,7 +211,7 @@ def run_ours(args):
         for i, c in enumerate(codecs):
             if record is not None:
                 record[0][i][0].record()
-            c.compress(dev_x[i], seed=0)
+            c.compress(dev_x[i], seed=0, flags=args.compress_flags)
             if record is not None:
                 record[0][i][1].record()
         for i, c in enumerate(codecs):
@@ -259,7 +259,7 @@ def run_ours(args):
     def e2e_step():
         for i, c in enumerate(codecs):
             dev_x[i].copy_(host_x[i], non_blocking=True)
-            c.compress(dev_x[i], seed=0)
+            c.compress(dev_x[i], seed=0, flags=args.compress_flags)
             c.decompress(out=dev_out[i])
             host_out[i].copy_(dev_out[i], non_blocking=True)
 
@@ -340,6 +340,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
+    ap.add_argument("--compress-flags", type=int, default=0,
+                    help="DIV_FLAG_* bits passed to div_compress_ex (profiling aid: 4 = strip ring kernel instead of the lagged one)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
