@@ -180,22 +180,33 @@ decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
 // flat kernel: any W and B, sample size a multiple of 4 elements, planes of at most FLAT_MAX_HW
 // elements.  One thread produces QPT quads of 4 consecutive elements (global flat order), which may
 // lie in different tiles, rows or planes: the tile of every position of a plane comes from a table
-// in shared memory (built once per CTA), the plane index advances with the position.
-// grid = (ceil(quads_per_sample / (256*QPT)), N), dynamic shared memory = 2 * HW bytes
+// in shared memory (built once per CTA), the plane index advances with the position; the low-frequency
+// values of the planes a CTA touches are staged in shared memory too.
+// grid = (ceil(quads_per_sample / (256*QPT)), N), dynamic shared memory = flat_smem_bytes()
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t FLAT_MAX_HW = 8192;
 
 struct DecFlat {
     uint32_t qps;        // quads per sample = CHW / 4
     uint32_t C, TPP, Wb, HW, W, B;
+    uint32_t table_words;    // 32-bit words the tile table takes in shared memory
+    uint32_t planes_per_cta; // upper bound of the planes one CTA touches
     FastDiv by_hw, by_w, by_b;
 };
+// planes a run of `elems` consecutive elements can touch, and the dynamic shared memory of the flat kernels
+inline uint32_t flat_planes_per_cta(uint32_t elems, uint32_t hw) { return (elems + hw - 1) / hw + 1; }
+inline uint32_t flat_table_words(uint32_t hw) { return (hw + 1) / 2; }
+inline size_t flat_smem_bytes(uint32_t elems, uint32_t hw, uint32_t tpp) {
+    return 4ull * flat_table_words(hw) + 4ull * flat_planes_per_cta(elems, hw) * tpp;
+}
 
 template <typename XT, typename LT, int Q, int QPT>
 __global__ void __launch_bounds__(256)
 decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFlat d) {
-    extern __shared__ uint16_t tile_of[];      // position inside a plane -> tile inside the plane
+    extern __shared__ uint32_t flat_smem[];
+    uint16_t* tile_of = reinterpret_cast<uint16_t*>(flat_smem);      // position inside a plane -> tile inside the plane
+    float* lfc_s = reinterpret_cast<float*>(flat_smem + d.table_words);   // low-frequency values of this CTA's planes
     __shared__ DeqTable<Q> table;
     const uint32_t n = blockIdx.y;
     table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
@@ -203,9 +214,13 @@ decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
         const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
         tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
     }
+    const uint32_t e_first = blockIdx.x * (1024u * QPT);
+    const uint32_t plane0 = fdiv(e_first, d.by_hw);
+    const uint32_t nplanes = min(d.planes_per_cta, d.C - plane0);
+    const LT* lfc_n = lfc + ((size_t)n * d.C + plane0) * d.TPP;
+    for (uint32_t idx = threadIdx.x; idx < nplanes * d.TPP; idx += 256u) lfc_s[idx] = Elem<LT>::load(lfc_n + idx);
     __syncthreads();
     const uint64_t sample_quad0 = (uint64_t)n * d.qps;
-    const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
     const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
 #pragma unroll
     for (int k = 0; k < QPT; ++k) {
@@ -213,16 +228,16 @@ decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
         if (q < d.qps) {
             const float4 hq = table.quad(quad_bits<Q>(packed, sample_quad0 + q));
             const float hv[4] = {hq.x, hq.y, hq.z, hq.w};
-            uint32_t plane = fdiv(q * 4u, d.by_hw);
+            const uint32_t plane = fdiv(q * 4u, d.by_hw);
             uint32_t rem = q * 4u - plane * d.HW;
-            const LT* lfc_p = lfc_n + (size_t)plane * d.TPP;
+            const float* lp = lfc_s + (plane - plane0) * d.TPP;
             float v[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                v[i] = __fadd_rn(Elem<LT>::load(lfc_p + tile_of[rem]), hv[i]);
+                v[i] = __fadd_rn(lp[tile_of[rem]], hv[i]);
                 if (++rem == d.HW) {
                     rem = 0;
-                    lfc_p += d.TPP;
+                    lp += d.TPP;
                 }
             }
             Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, v[0], v[1], v[2], v[3]);

@@ -150,7 +150,8 @@ bool decompress_fast_ok(const Shape& s) {
     return (s.W % 4 == 0) && s.B >= 4 && (s.B & (s.B - 1)) == 0 && s.N <= 65535;
 }
 bool decompress_flat_ok(const Shape& s) {
-    return (s.CHW % 4 == 0) && s.HW <= FLAT_MAX_HW && s.TPP <= 65535 && s.N <= 65535 && s.CHW < (1u << 31);
+    return (s.CHW % 4 == 0) && s.HW <= FLAT_MAX_HW && s.TPP <= 65535 && s.N <= 65535 && s.CHW < (1u << 31) &&
+           flat_smem_bytes(4u * 256u * DEC_QPT, s.HW, s.TPP) <= 40000;
 }
 
 }  // namespace
@@ -357,8 +358,11 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 d.by_w = make_fastdiv(s.W);
                 d.by_b = make_fastdiv(s.B);
                 const uint32_t per_block = 256u * DEC_QPT;
+                d.table_words = flat_table_words(s.HW);
+                d.planes_per_cta = flat_planes_per_cta(4u * per_block, s.HW);
                 dim3 grid((d.qps + per_block - 1) / per_block, s.N);
-                decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 2u * s.HW, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+                decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, flat_smem_bytes(4u * per_block, s.HW, s.TPP), stream>>>(
+                    lfc, packed, stats, (XT*)xhat_dev, d);
             } else {
                 const uint64_t g = (nwords + 255) / 256;
                 if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;

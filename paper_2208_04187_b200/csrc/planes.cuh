@@ -17,6 +17,7 @@
 // memory, the arithmetic of Eq. 9 runs on packed pairs.
 #pragma once
 
+#include "decompress.cuh"   // flat_table_words, flat_planes_per_cta, flat_smem_bytes
 #include "fused_v.cuh"
 
 namespace divk {
@@ -27,6 +28,8 @@ struct PlaneGeom {
     uint32_t planes_per_warp;     // 32 / lanes_per_plane
     uint32_t groups;              // ceil(C / planes_per_warp): warp passes per sample
     uint32_t qps;                 // quads per sample = CHW / 4
+    uint32_t table_words;         // 32-bit words the tile table takes in shared memory
+    uint32_t planes_per_cta;      // upper bound of the planes one CTA of the quantise kernel touches
     FastDiv by_hw, by_w, by_b;
 };
 
@@ -55,7 +58,10 @@ plane_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
             float sum = tree8<P2>(v);
 #pragma unroll
             for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-            const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
+            // one lane per tile divides, the others take its result
+            float mean = 0.f;
+            if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
+            mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
             const float stored = Elem<LT>::round(mean);
             if (ok) {
                 if (cw == 0) Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
@@ -87,13 +93,21 @@ __global__ void __launch_bounds__(256)
 plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const uint32_t* __restrict__ ws,
                    void* __restrict__ packed_v, float* __restrict__ stats, PlaneGeom g, uint64_t seed) {
     typedef typename PackedUnit<Q>::type OutT;
-    extern __shared__ uint16_t tile_of[];      // position inside a plane -> tile inside the plane
+    extern __shared__ uint32_t plane_smem[];
+    uint16_t* tile_of = reinterpret_cast<uint16_t*>(plane_smem);          // position inside a plane -> tile inside the plane
+    float* lfc_s = reinterpret_cast<float*>(plane_smem + g.table_words);  // stored low-frequency values of this CTA's planes
+    const uint32_t n = blockIdx.y;
     for (uint32_t idx = threadIdx.x; idx < g.HW; idx += 256u) {
         const uint32_t h = fdiv(idx, g.by_w), w = idx - h * g.W;
         tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * g.Wb + fdiv(w, g.by_b));
     }
+    const uint32_t plane0 = fdiv(blockIdx.x * (1024u * QPT), g.by_hw);
+    const uint32_t nplanes = min(g.planes_per_cta, g.C - plane0);
+    {
+        const LT* src = lfc + ((size_t)n * g.C + plane0) * g.TPP;
+        for (uint32_t idx = threadIdx.x; idx < nplanes * g.TPP; idx += 256u) lfc_s[idx] = Elem<LT>::load(src + idx);
+    }
     __syncthreads();
-    const uint32_t n = blockIdx.y;
     const uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
     const QParams qp = make_qparams(key_float(~__ldg(slot + 0)), key_float(__ldg(slot + 1)), Q);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -104,7 +118,6 @@ plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const u
     const uint64_t base = rng_sample_base(seed, n);
     const uint64_t sample_quad0 = (uint64_t)n * g.qps;
     const XT* x_n = x + (size_t)n * g.CHW;
-    const LT* lfc_n = lfc + (size_t)n * g.C * g.TPP;
     OutT* packed = reinterpret_cast<OutT*>(packed_v);
     const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
 #pragma unroll
@@ -113,13 +126,13 @@ plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const u
         if (q < g.qps) {
             uint64_t xy, zw;
             StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy, zw);
-            uint32_t plane = fdiv(q * 4u, g.by_hw);
+            const uint32_t plane = fdiv(q * 4u, g.by_hw);
             uint32_t rem = q * 4u - plane * g.HW;
-            const LT* lfc_p = lfc_n + (size_t)plane * g.TPP;
+            const float* lfc_p = lfc_s + (plane - plane0) * g.TPP;
             float lf[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                lf[i] = Elem<LT>::load(lfc_p + tile_of[rem]);
+                lf[i] = lfc_p[tile_of[rem]];
                 if (++rem == g.HW) {
                     rem = 0;
                     lfc_p += g.TPP;
@@ -154,6 +167,9 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
     g.planes_per_warp = 32u / g.lanes_per_plane;
     g.groups = (s.C + g.planes_per_warp - 1) / g.planes_per_warp;
     g.qps = s.CHW / 4;
+    g.table_words = flat_table_words(s.HW);
+    g.planes_per_cta = flat_planes_per_cta(4u * 256u * PLANE_QPT, s.HW);
+    if (flat_smem_bytes(4u * 256u * PLANE_QPT, s.HW, s.TPP) > 44000) return false;
     g.by_hw = host_fastdiv(s.HW);
     g.by_w = host_fastdiv(s.W);
     g.by_b = host_fastdiv(s.B);
@@ -183,7 +199,7 @@ inline div_status compress_planes_t(const div_desc* d, const Shape& s, const div
     if (cudaGetLastError() != cudaSuccess) return DIV_ERR_CUDA;
     const uint32_t per_block = 256u * PLANE_QPT;
     const dim3 grid2((g.qps + per_block - 1) / per_block, s.N);
-    const size_t smem = 2u * s.HW;
+    const size_t smem = flat_smem_bytes(4u * per_block, s.HW, s.TPP);
     void* packed = blob + lo.packed_off;
     float* stats = (float*)(blob + lo.stats_off);
     switch (d->qbits) {
