@@ -224,6 +224,11 @@ __device__ __forceinline__ uint64_t fma2_rn(uint64_t a, uint64_t b, uint64_t c) 
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
+__device__ __forceinline__ uint64_t fma2_rp(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
 
 // a staged strip row as two packed pairs (x, y) and (z, w), widened to fp32
 template <typename XT> struct StripRow2;
@@ -243,7 +248,12 @@ template <> struct StripRow2<__nv_bfloat16> {
 };
 
 // Codes of two elements sharing the 32-bit half `h` of a random word (Eq. 9 with stochastic
-// rounding), same arithmetic as quant_bits(): returns the two results MAGIC_CEIL_BITS + code.
+// rounding); returns the two results QUANT2_BITS + code.  Same integer as quant_bits(): with
+// F = 2^23 + field (the field dropped into the mantissa of 2^23), F * -2^-16 = -128 - u exactly, so one
+// fused multiply-add rounded towards +inf gives d = RU(t - u - 128), and ceil(d) = ceil(t - u) - 128
+// (rounding up never carries a value across an integer); the second add, rounded up onto the integer
+// grid of [2^23, 2^24), leaves that integer in the low mantissa bits.
+constexpr uint32_t QUANT2_BITS = MAGIC_CEIL_BITS - 128u;
 __device__ __forceinline__ void quant2(uint64_t x01, uint64_t stored2, uint64_t delta2, uint64_t scale2, float qmax,
                                        uint32_t h, uint32_t& b0, uint32_t& b1) {
     const uint64_t t01 = mul2_rn(sub2_rn(sub2_rn(x01, stored2), delta2), scale2);
@@ -251,10 +261,8 @@ __device__ __forceinline__ void quant2(uint64_t x01, uint64_t stored2, uint64_t 
     upk2(t01, t0, t1);
     t0 = fminf(t0, qmax);
     t1 = fminf(t1, qmax);
-    // 2^23 + field as a float: the 16-bit field in the low mantissa bits
-    const uint64_t f01 = sub2_rn(pk2u(__byte_perm(h, 0x4B000000u, 0x7610), __byte_perm(h, 0x4B000000u, 0x7632)),
-                                 pk2(8388608.0f, 8388608.0f));                                       // exact
-    const uint64_t d01 = fma2_rn(f01, pk2(-1.52587890625e-05f, -1.52587890625e-05f), pk2(t0, t1));   // fl(t - u)
+    const uint64_t f01 = pk2u(__byte_perm(h, 0x4B000000u, 0x7610), __byte_perm(h, 0x4B000000u, 0x7632));   // 2^23 + field
+    const uint64_t d01 = fma2_rp(f01, pk2(-1.52587890625e-05f, -1.52587890625e-05f), pk2(t0, t1));         // RU(t - u - 128)
     upk2u(add2_rp(d01, pk2(MAGIC_CEIL, MAGIC_CEIL)), b0, b1);
 }
 
@@ -266,7 +274,7 @@ __device__ __forceinline__ uint32_t quant_row(uint64_t xy, uint64_t zw, uint64_t
     uint32_t b0, b1, b2, b3;
     quant2(xy, stored2, delta2, scale2, qmax, (uint32_t)z, b0, b1);
     quant2(zw, stored2, delta2, scale2, qmax, (uint32_t)(z >> 32), b2, b3);
-    constexpr uint32_t BIAS = MAGIC_CEIL_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
+    constexpr uint32_t BIAS = QUANT2_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
     return b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS;
 }
 

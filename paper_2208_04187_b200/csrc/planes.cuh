@@ -143,7 +143,7 @@ plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const u
             uint32_t b0, b1, b2, b3;
             quant2(xy, pk2(lf[0], lf[1]), delta2, scale2, qmax, (uint32_t)z, b0, b1);
             quant2(zw, pk2(lf[2], lf[3]), delta2, scale2, qmax, (uint32_t)(z >> 32), b2, b3);
-            constexpr uint32_t BIAS = MAGIC_CEIL_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
+            constexpr uint32_t BIAS = QUANT2_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
             packed[sample_quad0 + q] = (OutT)(b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS);
         }
     }
