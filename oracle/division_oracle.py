@@ -21,7 +21,9 @@ What the method computes (DIVISION, Sec. 4.1 "Activation Map Compression" and Se
 
 Readings of points the paper leaves open (every one is also listed in the design notes):
 
-  * quantisation group: one (delta, Delta) pair per sample (all C*H*W residuals of it);
+  * quantisation group: one (delta, Delta) pair per sample (all C*H*W residuals of it); the
+    variant with one bfloat16 pair per (sample, channel) plane, which is what the paper's byte
+    count of Theorem 3A assumes, is stated in the last section of this file;
   * H or W not divisible by B: ceil grid, a partial tile is averaged over its in-bounds
     elements (this reproduces the paper's "N < B gives a 1x1 low-frequency map" rule);
   * the residual is taken against the STORED (rounded) low-frequency value, so that the
@@ -386,3 +388,152 @@ def parse_blob(blob: np.ndarray, n: int, c: int, h: int, w: int, block: int, qbi
     codes = unpack_codes(words, qbits, n * c * h * w).reshape(n, c * h * w)
     return Compressed((n, c, h, w), block, qbits, x_dtype, lfc_dtype, lfc, codes, words,
                       stats[:, 0].copy(), stats[:, 1].copy(), lo)
+
+
+# ----------------------------------------------------------------------------------------
+# per-plane quantisation groups with bfloat16 (delta, Delta)
+# ----------------------------------------------------------------------------------------
+# The paper counts N^2*Q/8 + 4 bytes per channel plane for the high-frequency component
+# (proof of Theorem 3A) and says that Delta and delta are cached in bfloat16 (Sec. 4.1): one
+# (delta, Delta) pair of two bfloat16 numbers per (sample, channel) plane.  This section states
+# that variant.  Everything else (pooling, residual against the stored low-frequency value,
+# stochastic rounding, DIVRNG-v1, packing order) is as above.
+#
+# Reading for the bfloat16 rounding, on which the paper is silent: a delta rounded to NEAREST
+# could land above the true minimum and make (h - delta)/Delta negative, and a Delta rounded
+# down could push the largest code past 2^Q - 1.  So
+#     delta_b = the largest bfloat16 number <= min H^H          (rounded down)
+#     Delta_b = the smallest bfloat16 number >= (max H^H - delta_b) / (2^Q - 1)   (rounded up)
+# and both the encoder and the decoder use exactly these stored numbers:
+#     t = (h - delta_b) * (1 / Delta_b),   h_hat = Delta_b * code + delta_b.
+# Then 0 <= t <= (2^Q - 1) up to fp32 rounding (the clamp of Eq. 9's range only absorbs that),
+# |h_hat - h| <= Delta_b, and E[h_hat] = h as in Sec. 4.1.  A zero is stored as +0.0.  A plane whose
+# Delta_b or 1/Delta_b is zero or not finite is degenerate: Delta_b = 0 is stored, every code is 0
+# (and delta_b = 0 too when the minimum lies below the most negative finite bfloat16 number).
+def bf16_floor_bits(a: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns of the largest bfloat16 numbers <= a (finite fp32 input)."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    hi = u >> np.uint64(16)
+    inexact = (u & np.uint64(0xFFFF)) != 0
+    hi = hi + (inexact & (a < 0)).astype(np.uint64)      # truncation moves a negative number up
+    hi = np.where(a == 0, np.uint64(0), hi)
+    return hi.astype(np.uint16)
+
+
+def bf16_ceil_bits(a: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns of the smallest bfloat16 numbers >= a (finite fp32 input)."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    hi = u >> np.uint64(16)
+    inexact = (u & np.uint64(0xFFFF)) != 0
+    hi = hi + (inexact & (a > 0)).astype(np.uint64)      # truncation moves a positive number down
+    hi = np.where(a == 0, np.uint64(0), hi)
+    return hi.astype(np.uint16)
+
+
+def plane_stats(r_plane: np.ndarray, qbits: int):
+    """(delta_b, Delta_b, scale) of one (sample, channel) plane, all as fp32 values (rule above)."""
+    qmax = np.float32((1 << qbits) - 1)
+    low = np.float32(r_plane.min())
+    top = np.float32(r_plane.max())
+    delta_b = bf16_bits_to_f32(bf16_floor_bits(np.array([low])))[0]
+    zero = np.float32(0)
+    if not np.isfinite(delta_b):                       # minimum below the most negative bfloat16 number
+        return zero, zero, zero
+    with np.errstate(over="ignore", divide="ignore", invalid="ignore"):
+        rng = np.float32(top - delta_b)
+        step = np.float32(rng / qmax)
+        step_b = bf16_bits_to_f32(bf16_ceil_bits(np.array([step])))[0] if np.isfinite(step) else np.float32(np.inf)
+        scale = np.float32(np.float32(1) / step_b) if step_b > 0 else zero
+    if not (np.isfinite(step_b) and step_b > 0 and np.isfinite(scale) and scale > 0):
+        return delta_b, zero, zero
+    return delta_b, step_b, scale
+
+
+def plane_layout(n: int, c: int, h: int, w: int, block: int, qbits: int,
+                 x_dtype: str = F32, lfc_dtype: str = F32) -> Layout:
+    """As compressed_layout, but the stats section holds N*C pairs of bfloat16: 4 bytes per plane."""
+    lo = compressed_layout(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
+    stats_bytes = 4 * n * c
+    return Layout(lo.lfc_off, lo.lfc_bytes, lo.packed_off, lo.packed_bytes, lo.stats_off, stats_bytes,
+                  lo.stats_off + stats_bytes, lo.lfc_bytes + lo.packed_bytes + stats_bytes, lo.raw_bytes)
+
+
+@dataclass
+class PlaneCompressed:
+    shape: tuple
+    block: int
+    qbits: int
+    x_dtype: str
+    lfc_dtype: str
+    lfc: np.ndarray        # [N,C,Hb,Wb] fp32 values as stored
+    codes: np.ndarray      # [N, C, H*W] uint8
+    words: np.ndarray      # packed uint32 words (same element order as the per-sample form)
+    delta: np.ndarray      # [N, C] fp32 values of the stored bfloat16 delta_b
+    step: np.ndarray       # [N, C] fp32 values of the stored bfloat16 Delta_b
+    layout: Layout
+
+    def blob(self) -> np.ndarray:
+        out = np.zeros(self.layout.total_bytes, dtype=np.uint8)
+        if self.lfc_dtype == F32:
+            lfc_raw = self.lfc.astype("<f4").tobytes()
+        else:
+            lfc_raw = f32_to_bf16_bits(self.lfc).astype("<u2").tobytes()
+        lo = self.layout
+        out[lo.lfc_off:lo.lfc_off + lo.lfc_bytes] = np.frombuffer(lfc_raw, dtype=np.uint8)
+        out[lo.packed_off:lo.packed_off + lo.packed_bytes] = np.frombuffer(
+            self.words.astype("<u4").tobytes(), dtype=np.uint8)
+        pair = np.stack([f32_to_bf16_bits(self.delta.reshape(-1)),       # exact: the values are bfloat16
+                         f32_to_bf16_bits(self.step.reshape(-1))], axis=1).astype("<u2")
+        out[lo.stats_off:lo.stats_off + lo.stats_bytes] = np.frombuffer(pair.tobytes(), dtype=np.uint8)
+        return out
+
+
+def compress_planes(x: np.ndarray, block: int, qbits: int, seed: int,
+                    x_dtype: str = F32, lfc_dtype: str = F32, first_sample: int = 0) -> PlaneCompressed:
+    """The forward-loop steps of Algorithm 1 with one quantisation group per (sample, channel) plane."""
+    if qbits not in SUPPORTED_QBITS:
+        raise ValueError("Q must divide 32")
+    x32 = widen_input(x, x_dtype)
+    n, c, h, w = x32.shape
+    hw = h * w
+    lfc = round_to_dtype(lfc_mean_f32(x32, block), lfc_dtype)
+    r = (x32 - upsample_nearest(lfc, block, h, w)).reshape(n, c, hw)
+    codes = np.empty((n, c, hw), dtype=np.uint8)
+    delta = np.empty((n, c), dtype=np.float32)
+    step = np.empty((n, c), dtype=np.float32)
+    for i in range(n):
+        fields = divrng_fields(seed, first_sample + i, np.arange(c * hw, dtype=np.uint64)).reshape(c, hw)
+        for j in range(c):                                               # Quant, per plane
+            delta[i, j], step[i, j], scale = plane_stats(r[i, j], qbits)
+            codes[i, j] = quantize(r[i, j], delta[i, j], scale, fields[j], qbits)
+    words = pack_codes(codes.reshape(-1), qbits)
+    layout = plane_layout(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
+    return PlaneCompressed((n, c, h, w), block, qbits, x_dtype, lfc_dtype, lfc, codes, words, delta, step, layout)
+
+
+def decompress_planes(comp: PlaneCompressed) -> np.ndarray:
+    """The backward-loop steps of Algorithm 1 for per-plane groups; fp32 values rounded to the activation dtype."""
+    n, c, h, w = comp.shape
+    codes = unpack_codes(comp.words, comp.qbits, n * c * h * w).reshape(n, c, h * w)
+    hh = (comp.step[:, :, None].astype(np.float32) * codes.astype(np.float32)
+          + comp.delta[:, :, None].astype(np.float32)).astype(np.float32)
+    xhat = upsample_nearest(comp.lfc, comp.block, h, w) + hh.reshape(n, c, h, w)
+    return round_to_dtype(xhat.astype(np.float32), comp.x_dtype)
+
+
+def parse_plane_blob(blob: np.ndarray, n: int, c: int, h: int, w: int, block: int, qbits: int,
+                     x_dtype: str = F32, lfc_dtype: str = F32) -> PlaneCompressed:
+    """Read a per-plane compressed buffer back into its parts."""
+    lo = plane_layout(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    hb, wb = grid_shape(h, w, block)
+    raw = blob[lo.lfc_off:lo.lfc_off + lo.lfc_bytes]
+    lfc = raw.view("<f4").astype(np.float32) if lfc_dtype == F32 else bf16_bits_to_f32(raw.view("<u2"))
+    lfc = lfc.reshape(n, c, hb, wb)
+    words = blob[lo.packed_off:lo.packed_off + lo.packed_bytes].view("<u4").astype(np.uint32)
+    pair = blob[lo.stats_off:lo.stats_off + lo.stats_bytes].view("<u2").reshape(n, c, 2)
+    codes = unpack_codes(words, qbits, n * c * h * w).reshape(n, c, h * w)
+    return PlaneCompressed((n, c, h, w), block, qbits, x_dtype, lfc_dtype, lfc, codes, words,
+                           bf16_bits_to_f32(pair[:, :, 0].copy()), bf16_bits_to_f32(pair[:, :, 1].copy()), lo)
