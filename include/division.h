@@ -201,6 +201,33 @@ div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, v
                                       void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream,
                                       uint32_t flags, uint64_t timeout_ns);
 
+/*
+ * Per-plane quantisation groups: the same pair of operations with one (delta, Delta) pair per
+ * (sample, channel) plane, stored as two bfloat16 numbers.  This is the grouping behind the paper's count of
+ * N^2*Q/8 + 4 bytes per channel for the high-frequency component (Sec. 4.1; proof of Theorem 3A), and
+ * "Delta and delta are cached in bfloat16" (Sec. 4.1).  Differences from div_compress / div_decompress:
+ *   - blob: same sections, but stats = N*C little-endian 32-bit words, low half delta_b, high half Delta_b
+ *     (bfloat16 bit patterns); closed form = lfc + packed + 4*N*C bytes; layout.workspace_bytes = 0;
+ *   - rounding of the pair, on which the paper is silent: delta_b = largest bfloat16 number <= min H^H,
+ *     Delta_b = smallest bfloat16 number >= (max H^H - delta_b)/(2^Q - 1); both sides use the stored pair:
+ *     t = (H^H - delta_b) * (1/Delta_b), H^H_hat = Delta_b * V^H + delta_b.  A plane whose Delta_b or
+ *     1/Delta_b would be zero or not finite stores Delta_b = 0 and all codes 0;
+ *   - a plane's extremes stay inside one CTA, so compress needs no scratch and no device-side waiting;
+ *   - n*c < 2^31 (else DIV_ERR_SHAPE).
+ * Everything else (pooling grid, residual against the stored value, stochastic rounding, random stream,
+ * packing order, argument meaning, ownership, error codes) is as documented above.
+ * flags: 0, or DIV_FLAG_FORCE_TWO_PASS to take the general kernel (one CTA per plane) even where the
+ * register-resident strip kernel applies (W%4==0, B in {4,8}, Q in {2,4,8}, planes of at most 512 strips of
+ * 4 columns x B rows).
+ */
+div_status div_planegroup_bytes(const div_desc* desc, div_layout* out);
+div_status div_planegroup_compress(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                                   uint64_t seed, void* cuda_stream, uint32_t flags);
+div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes,
+                                     void* xhat_dev, void* cuda_stream);
+/* plan.fused: 1 strip kernel, 0 general kernel; plan.decompress_fast: 1 quad kernel, 0 general. */
+div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
+
 /* Which kernels a descriptor maps to on the current device.  desc, out: host. */
 div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
 

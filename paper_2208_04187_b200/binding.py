@@ -24,6 +24,7 @@ DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 EXPORTED_SYMBOLS = (
     "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_debug_compress_starved",
     "div_decompress", "div_plan_query",
+    "div_planegroup_bytes", "div_planegroup_compress", "div_planegroup_decompress", "div_planegroup_plan_query",
     "div_read_device_status", "div_status_string",
 )
 
@@ -78,6 +79,15 @@ def lib() -> ctypes.CDLL:
         L.div_decompress.restype = c_int32
         L.div_plan_query.argtypes = [ctypes.POINTER(DivDesc), c_uint32, ctypes.POINTER(DivPlan)]
         L.div_plan_query.restype = c_int32
+        L.div_planegroup_bytes.argtypes = [ctypes.POINTER(DivDesc), ctypes.POINTER(DivLayout)]
+        L.div_planegroup_bytes.restype = c_int32
+        L.div_planegroup_compress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_void_p, c_size_t, c_uint64, c_void_p,
+                                              c_uint32]
+        L.div_planegroup_compress.restype = c_int32
+        L.div_planegroup_decompress.argtypes = L.div_decompress.argtypes
+        L.div_planegroup_decompress.restype = c_int32
+        L.div_planegroup_plan_query.argtypes = L.div_plan_query.argtypes
+        L.div_planegroup_plan_query.restype = c_int32
         L.div_read_device_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_int32)]
         L.div_read_device_status.restype = c_int32
         L.div_status_string.argtypes = [c_int32]
@@ -141,6 +151,33 @@ def div_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xhat_ptr: int,
     _check(st, "div_decompress")
 
 
+def div_planegroup_bytes(desc: DivDesc) -> DivLayout:
+    """Layout of the per-plane form: one bfloat16 (delta, Delta) pair per (sample, channel) plane."""
+    out = DivLayout()
+    _check(lib().div_planegroup_bytes(ctypes.byref(desc), ctypes.byref(out)), "div_planegroup_bytes")
+    return out
+
+
+def div_planegroup_plan_query(desc: DivDesc, flags: int = 0) -> DivPlan:
+    out = DivPlan()
+    _check(lib().div_planegroup_plan_query(ctypes.byref(desc), int(flags), ctypes.byref(out)),
+           "div_planegroup_plan_query")
+    return out
+
+
+def div_planegroup_compress(desc: DivDesc, x_ptr: int, comp_ptr: int, comp_capacity: int, seed: int,
+                            stream: int = 0, flags: int = 0) -> None:
+    st = lib().div_planegroup_compress(ctypes.byref(desc), c_void_p(x_ptr), c_void_p(comp_ptr), comp_capacity,
+                                       c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream), int(flags))
+    _check(st, "div_planegroup_compress")
+
+
+def div_planegroup_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xhat_ptr: int, stream: int = 0) -> None:
+    st = lib().div_planegroup_decompress(ctypes.byref(desc), c_void_p(comp_ptr), comp_bytes, c_void_p(xhat_ptr),
+                                         c_void_p(stream))
+    _check(st, "div_planegroup_decompress")
+
+
 def div_read_device_status(ws_ptr: int, stream: int = 0) -> int:
     out = c_int32(0)
     _check(lib().div_read_device_status(c_void_p(ws_ptr), c_void_p(stream), ctypes.byref(out)),
@@ -202,3 +239,37 @@ class Codec:
 
     def device_status(self) -> int:
         return div_read_device_status(self.workspace.data_ptr(), current_stream_handle())
+
+
+class PlaneGroupCodec:
+    """Codec with one bfloat16 (delta, Delta) pair per (sample, channel) plane; no workspace."""
+
+    def __init__(self, n, c, h, w, block, qbits, x_dtype="f32", lfc_dtype="f32", device="cuda"):
+        torch = _torch()
+        self.x_dtype, self.lfc_dtype = x_dtype, lfc_dtype
+        self.desc = make_desc(n, c, h, w, block, qbits, x_dtype, lfc_dtype)
+        self.layout = div_planegroup_bytes(self.desc)
+        self.shape = (n, c, h, w)
+        self.device = torch.device(device)
+        self.blob = torch.zeros(int(self.layout.total_bytes), dtype=torch.uint8, device=self.device)
+
+    def plan(self, flags: int = 0) -> DivPlan:
+        return div_planegroup_plan_query(self.desc, flags)
+
+    def compress(self, x, seed: int = 0, flags: int = 0, blob=None):
+        torch = _torch()
+        blob = self.blob if blob is None else blob
+        if not (x.is_cuda and x.is_contiguous() and tuple(x.shape) == self.shape
+                and x.dtype == torch_dtype(self.x_dtype)):
+            raise ValueError("x must be a contiguous CUDA tensor matching the descriptor")
+        div_planegroup_compress(self.desc, x.data_ptr(), blob.data_ptr(), blob.numel(), seed,
+                                current_stream_handle(), flags)
+        return blob
+
+    def decompress(self, blob=None, out=None):
+        torch = _torch()
+        blob = self.blob if blob is None else blob
+        if out is None:
+            out = torch.empty(self.shape, dtype=torch_dtype(self.x_dtype), device=self.device)
+        div_planegroup_decompress(self.desc, blob.data_ptr(), blob.numel(), out.data_ptr(), current_stream_handle())
+        return out

@@ -12,6 +12,7 @@
 #include "fused.cuh"
 #include "fused_v.cuh"
 #include "lagged.cuh"
+#include "planegroup.cuh"
 #include "planes.cuh"
 #include "twopass.cuh"
 
@@ -75,6 +76,17 @@ void make_layout(const div_desc* d, const Shape& s, div_layout* out) {
     out->raw_bytes = s.total * dtype_bytes(d->x_dtype);
     out->workspace_bytes = align_up(4ull * (WS_HEADER_WORDS + (uint64_t)WS_SLOT_WORDS * s.N), 256);
 }
+
+// per-plane groups: the same sections, but the stats section holds one bfloat16 pair (4 bytes) per plane and
+// no scratch is needed
+void make_layout_pg(const div_desc* d, const Shape& s, div_layout* out) {
+    make_layout(d, s, out);
+    out->stats_bytes = 4ull * s.N * s.C;
+    out->total_bytes = out->stats_off + out->stats_bytes;
+    out->closed_form_bytes = out->lfc_bytes + out->packed_bytes + out->stats_bytes;
+    out->workspace_bytes = 0;
+}
+inline bool pg_shape_ok(const Shape& s) { return (uint64_t)s.N * s.C < (1ull << 31); }
 
 FastDiv make_fastdiv(uint32_t d) {
     FastDiv f;
@@ -426,6 +438,126 @@ div_status div_compress_static(const div_desc* desc, const void* x_dev, void* co
     if (got != DIV_OK) return got;
     // same path as div_compress from here on (it clears the part of the scratch it uses on the stream)
     return div_compress_ex(desc, x_dev, comp_dev, comp_capacity, ws, STATIC_WS_BYTES, seed, cuda_stream, 0u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-plane quantisation groups
+// ------------------------------------------------------------------------------------------------
+div_status div_planegroup_bytes(const div_desc* desc, div_layout* out) {
+    if (!desc || !out) return DIV_ERR_NULL;
+    const div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    const Shape s = make_shape(desc);
+    if (!pg_shape_ok(s)) return DIV_ERR_SHAPE;
+    make_layout_pg(desc, s, out);
+    return DIV_OK;
+}
+
+div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
+    if (!desc || !out) return DIV_ERR_NULL;
+    const div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    const Shape s = make_shape(desc);
+    if (!pg_shape_ok(s)) return DIV_ERR_SHAPE;
+    *out = div_plan();
+    PgPlan pl;
+    if (!(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_strip(desc, s, &pl)) {
+        out->fused = 1;
+        out->grid = pl.grid;
+        out->threads = PG_THREADS;
+        out->chunk_elems = (int64_t)pl.G * s.HW;
+        out->chunks_per_sample = (s.C + pl.G - 1) / pl.G;
+    } else {
+        out->fused = 0;
+        out->grid = (int32_t)(s.N * s.C);
+        out->threads = 256;
+        out->chunk_elems = s.HW;
+        out->chunks_per_sample = s.C;
+    }
+    out->decompress_fast = decompress_fast_ok(s) ? 1 : 0;
+    return DIV_OK;
+}
+
+div_status div_planegroup_compress(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                                   uint64_t seed, void* cuda_stream, uint32_t flags) {
+    if (!desc || !x_dev || !comp_dev) return DIV_ERR_NULL;
+    div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (flags & ~DIV_FLAG_FORCE_TWO_PASS) return DIV_ERR_PARAM;
+    if (!aligned16(x_dev) || !aligned16(comp_dev)) return DIV_ERR_ALIGN;
+    const Shape s = make_shape(desc);
+    if (!pg_shape_ok(s)) return DIV_ERR_SHAPE;
+    div_layout lo;
+    make_layout_pg(desc, s, &lo);
+    if (comp_capacity < lo.total_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    uint8_t* blob = (uint8_t*)comp_dev;
+    PgPlan pl;
+    if (!(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_strip(desc, s, &pl))
+        return compress_pg_strip(desc, s, lo, pl, x_dev, blob, seed, stream);
+    // general kernel: words shared by two planes (and the zero-padded last word) are merged with atomic ORs
+    // into a cleared buffer
+    if (((uint64_t)s.HW * (uint64_t)desc->qbits) % 32u != 0 &&
+        cudaMemsetAsync(blob + lo.packed_off, 0, lo.packed_bytes, stream) != cudaSuccess)
+        return DIV_ERR_CUDA;
+    return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+            pg_general_kernel<XT, LT, decltype(q)::value><<<s.N * s.C, 256, 0, stream>>>(
+                (const XT*)x_dev, (LT*)(blob + lo.lfc_off), (uint32_t*)(blob + lo.packed_off),
+                (uint32_t*)(blob + lo.stats_off), s, seed);
+            return launch_status();
+        });
+    });
+}
+
+div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes, void* xhat_dev,
+                                     void* cuda_stream) {
+    if (!desc || !comp_dev || !xhat_dev) return DIV_ERR_NULL;
+    div_status st = check_desc(desc);
+    if (st != DIV_OK) return st;
+    if (!aligned16(comp_dev) || !aligned16(xhat_dev)) return DIV_ERR_ALIGN;
+    const Shape s = make_shape(desc);
+    if (!pg_shape_ok(s)) return DIV_ERR_SHAPE;
+    div_layout lo;
+    make_layout_pg(desc, s, &lo);
+    if (comp_bytes < lo.total_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const uint8_t* blob = (const uint8_t*)comp_dev;
+    const uint64_t nwords = lo.packed_bytes / 4;
+    return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+            constexpr int Q = decltype(q)::value;
+            const LT* lfc = (const LT*)(blob + lo.lfc_off);
+            const uint32_t* packed = (const uint32_t*)(blob + lo.packed_off);
+            const uint32_t* stats = (const uint32_t*)(blob + lo.stats_off);
+            if (decompress_fast_ok(s)) {
+                DecFast d;
+                d.qps = s.CHW / 4;
+                d.C = s.C;
+                d.TPP = s.TPP;
+                d.Wb = s.Wb;
+                d.log2B = 0;
+                while ((1u << d.log2B) < s.B) ++d.log2B;
+                d.hwq = s.HW / 4;
+                d.wq = s.W / 4;
+                d.by_hwq = make_fastdiv(d.hwq);
+                d.by_wq = make_fastdiv(d.wq);
+                const uint32_t per_block = 256u * DEC_QPT;
+                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+            } else {
+                const uint64_t g = (nwords + 255) / 256;
+                if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
+                pg_decompress_general_kernel<XT, LT, Q><<<(unsigned)g, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, s, nwords);
+            }
+            return launch_status();
+        });
+    });
 }
 
 div_status div_read_device_status(const void* workspace_dev, void* cuda_stream, int32_t* out_status) {

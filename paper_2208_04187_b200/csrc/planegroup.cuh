@@ -1,0 +1,461 @@
+// Per-plane quantisation groups: one (delta, Delta) pair of two bfloat16 numbers per (sample, channel)
+// plane -- the grouping behind the paper's byte count of N^2*Q/8 + 4 bytes per channel (Sec. 4.1, proof
+// of Theorem 3A; "Delta and delta are cached in bfloat16").  Pooling, residual, stochastic rounding, the
+// random stream and the packing order are those of the per-sample kernels.
+//
+// Rounding of the pair (the paper is silent): delta_b is the largest bfloat16 number <= min H^H and
+// Delta_b the smallest bfloat16 number >= (max H^H - delta_b) / (2^Q - 1); encoder and decoder both use the
+// stored pair: t = (h - delta_b) * (1 / Delta_b), h_hat = Delta_b * code + delta_b.  So t never turns
+// negative and never passes 2^Q - 1 by more than a rounding error, which the clamp absorbs.
+//
+// A plane's extremes need no communication between CTAs here, so compress is a true single pass:
+//   pg_strip_kernel    W % 4 == 0, B in {4, 8}, Q in {2, 4, 8}, planes of at most PG_CAP strip slots: a CTA
+//                      takes a few whole planes; every thread keeps its strips (4 columns x B rows) in
+//                      registers from the load, through the tile means and the CTA-wide extremes, to the
+//                      quantiser.  x crosses HBM once and is never re-read from anywhere.
+//   pg_general_kernel  any shape: one CTA per plane, second read of the plane from L1/L2.
+#pragma once
+
+#include "decompress.cuh"
+#include "lagged.cuh"
+
+namespace divk {
+
+#ifndef DIVK_PG_THREADS
+#define DIVK_PG_THREADS 256
+#endif
+#ifndef DIVK_PG_SLOTS
+#define DIVK_PG_SLOTS 2
+#endif
+#ifndef DIVK_PG_MIN_CTAS
+#define DIVK_PG_MIN_CTAS 2
+#endif
+constexpr int PG_THREADS = DIVK_PG_THREADS;
+constexpr int PG_K = DIVK_PG_SLOTS;               // strip slots a thread keeps in registers
+constexpr uint32_t PG_CAP = PG_THREADS * PG_K;    // strip slots of one CTA
+
+// ------------------------------------------------------------------------------------------------
+// the bfloat16 pair of one plane
+// ------------------------------------------------------------------------------------------------
+struct PgQ {
+    float delta;   // delta_b as fp32
+    float step;    // Delta_b as fp32 (0: degenerate plane, every code 0)
+    float scale;   // 1 / Delta_b (0 when degenerate)
+};
+__device__ __forceinline__ bool f32_finite(float v) { return (__float_as_uint(v) & 0x7F800000u) != 0x7F800000u; }
+// largest bfloat16 number <= v / smallest bfloat16 number >= v, as fp32; a zero comes out as +0.0
+__device__ __forceinline__ float bf16_floor(float v) {
+    const uint32_t u = __float_as_uint(v);
+    uint32_t hi = u >> 16;
+    if ((u & 0xFFFFu) != 0u && v < 0.f) hi += 1u;     // cutting the low bits moves a negative number up
+    if (v == 0.f) hi = 0u;
+    return __uint_as_float(hi << 16);
+}
+__device__ __forceinline__ float bf16_ceil(float v) {
+    const uint32_t u = __float_as_uint(v);
+    uint32_t hi = u >> 16;
+    if ((u & 0xFFFFu) != 0u && v > 0.f) hi += 1u;     // cutting the low bits moves a positive number down
+    if (v == 0.f) hi = 0u;
+    return __uint_as_float(hi << 16);
+}
+__device__ __forceinline__ PgQ pg_params(float rmin, float rmax, int qbits) {
+    PgQ q = {0.f, 0.f, 0.f};
+    const float d = bf16_floor(rmin);
+    if (!f32_finite(d)) return q;                     // minimum below the most negative bfloat16 number
+    q.delta = d;
+    const float step = __fdiv_rn(__fsub_rn(rmax, d), (float)((1 << qbits) - 1));
+    if (!f32_finite(step)) return q;
+    const float sb = bf16_ceil(step);
+    if (!f32_finite(sb) || !(sb > 0.f)) return q;
+    const float sc = __fdiv_rn(1.0f, sb);
+    if (!f32_finite(sc) || !(sc > 0.f)) return q;
+    q.step = sb;
+    q.scale = sc;
+    return q;
+}
+// the stored pair: low half-word delta_b, high half-word Delta_b
+__device__ __forceinline__ uint32_t pg_stats_word(const PgQ& q) {
+    return (__float_as_uint(q.delta) >> 16) | (__float_as_uint(q.step) & 0xFFFF0000u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// strip kernel
+// ------------------------------------------------------------------------------------------------
+struct PgParams {
+    Shape s;
+    const void* x;
+    void* lfc;
+    void* packed;
+    uint32_t* stats;
+    uint64_t seed;
+    uint64_t rng_row_step;   // K_GROUP * (W / 4)
+    uint32_t planes;         // N * C
+    uint32_t spb, spp;       // strip slots per band and per plane
+    uint32_t G;              // planes per CTA
+    uint32_t tail_rows;      // rows of the last band of a plane
+    FastDiv by_spp, by_spb, by_c;
+    float inv_cnt[4];        // as in the lagged kernel: [tail row band][tail column tile]
+    float cnt[4];
+};
+
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(PG_THREADS, DIVK_PG_MIN_CTAS)
+pg_strip_kernel(const PgParams p) {
+    constexpr uint32_t LPT = P2 / 4;
+    typedef typename PackedUnit<Q>::type OutT;
+    __shared__ uint32_t s_key[2 * PG_CAP];     // per plane of this CTA: ~key(min), key(max)
+    __shared__ float s_par[2 * PG_CAP];        // per plane: delta_b, 1 / Delta_b
+
+    const Shape& s = p.s;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t row_bytes = s.W * (uint32_t)sizeof(XT);
+    const uint32_t W4 = s.W >> 2;
+    const uint32_t plane0 = blockIdx.x * p.G;
+    for (uint32_t i = tid; i < 2u * p.G; i += PG_THREADS) s_key[i] = 0u;
+
+    // ---- where this thread's slots are, and their loads (everything a thread reads is requested at once)
+    uint32_t rows[PG_K], pl[PG_K], first[PG_K], tile[PG_K], which[PG_K];
+    uint64_t vxy[PG_K][P2], vzw[PG_K][P2];
+#pragma unroll
+    for (int k = 0; k < PG_K; ++k) {
+        const uint32_t S = tid + (uint32_t)k * PG_THREADS;
+        pl[k] = fdiv(S, p.by_spp);
+        const uint32_t sl = S - pl[k] * p.spp;
+        const uint32_t bh = fdiv(sl, p.by_spb);
+        const uint32_t q = sl - bh * p.spb;
+        const bool ok = pl[k] < p.G && plane0 + pl[k] < p.planes && 4u * q < s.W;
+        rows[k] = ok ? ((bh + 1u == s.Hb) ? p.tail_rows : s.B) : 0u;
+        first[k] = bh * s.B * s.W + 4u * q;                  // first element of the slot inside its plane
+        tile[k] = bh * s.Wb + q / LPT;
+        const uint32_t tail_col = (q / LPT == s.Wb - 1u && (s.W % s.B) != 0u) ? 1u : 0u;
+        which[k] = ((rows[k] != s.B) ? 2u : 0u) + tail_col;
+        const unsigned char* xs = reinterpret_cast<const unsigned char*>(
+            reinterpret_cast<const XT*>(p.x) + ((size_t)(plane0 + (ok ? pl[k] : 0u)) * s.HW + first[k]));
+#pragma unroll
+        for (int r = 0; r < P2; ++r) {
+            if ((uint32_t)r < rows[k]) {
+                StripRow2<XT>::load(xs + (size_t)r * row_bytes, vxy[k][r], vzw[k][r]);
+            } else {
+                vxy[k][r] = 0ull;
+                vzw[k][r] = 0ull;
+            }
+        }
+    }
+    __syncthreads();      // the key slots are cleared
+
+    // ---- tile means (fixed summation order), stored low-frequency values, extremes of the residual
+    float stored[PG_K];
+#pragma unroll
+    for (int k = 0; k < PG_K; ++k) {
+        uint64_t cxy[P2], czw[P2];
+#pragma unroll
+        for (int r = 0; r < P2; ++r) {
+            cxy[r] = vxy[k][r];
+            czw[r] = vzw[k][r];
+        }
+#pragma unroll
+        for (int w = P2; w > 1; w >>= 1) {
+#pragma unroll
+            for (int i = 0; i < w / 2; ++i) {
+                cxy[i] = add2_rn(cxy[2 * i], cxy[2 * i + 1]);
+                czw[i] = add2_rn(czw[2 * i], czw[2 * i + 1]);
+            }
+        }
+        float c0, c1, c2, c3;
+        upk2(cxy[0], c0, c1);
+        upk2(czw[0], c2, c3);
+        float sum = __fadd_rn(__fadd_rn(c0, c1), __fadd_rn(c2, c3));
+#pragma unroll
+        for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+        const float inv = p.inv_cnt[which[k]];
+        const float mean = (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, p.cnt[which[k]]);
+        stored[k] = Elem<LT>::round(mean);
+        if (rows[k] != 0u) {
+            if ((tid % LPT) == 0u)
+                Elem<LT>::store(reinterpret_cast<LT*>(p.lfc) + ((size_t)(plane0 + pl[k]) * s.TPP + tile[k]), mean);
+            // extremes of x over the in-bounds rows; x -> fl(x - stored) is monotone
+            float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+#pragma unroll
+            for (int r = 0; r < P2; ++r) {
+                if ((uint32_t)r < rows[k]) {
+                    float a_, b_, c_, d_;
+                    upk2(vxy[k][r], a_, b_);
+                    upk2(vzw[k][r], c_, d_);
+                    blo = fmin3(blo, a_, b_);
+                    blo = fmin3(blo, c_, d_);
+                    bhi = fmax3(bhi, a_, b_);
+                    bhi = fmax3(bhi, c_, d_);
+                }
+            }
+            atomicMax(&s_key[2u * pl[k]], ~float_key(__fsub_rn(blo, stored[k])));
+            atomicMax(&s_key[2u * pl[k] + 1u], float_key(__fsub_rn(bhi, stored[k])));
+        }
+    }
+    __syncthreads();      // every plane's extremes are complete
+
+    for (uint32_t i = tid; i < p.G; i += PG_THREADS) {
+        if (plane0 + i < p.planes) {
+            const PgQ q = pg_params(key_float(~s_key[2u * i]), key_float(s_key[2u * i + 1u]), Q);
+            s_par[2u * i] = q.delta;
+            s_par[2u * i + 1u] = q.scale;
+            p.stats[plane0 + i] = pg_stats_word(q);
+        }
+    }
+    __syncthreads();
+
+    // ---- Eq. 9 on the values still held in registers
+#pragma unroll
+    for (int k = 0; k < PG_K; ++k) {
+        if (rows[k] != 0u) {
+            const uint32_t plane = plane0 + pl[k];
+            const uint32_t n = fdiv(plane, p.by_c);
+            const uint32_t c = plane - n * s.C;
+            const float delta = s_par[2u * pl[k]], scale = s_par[2u * pl[k] + 1u];
+            const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale), stored2 = pk2(stored[k], stored[k]);
+            const uint32_t e = c * s.HW + first[k];                         // in-sample index, a multiple of 4
+            uint64_t ctr = rng_sample_base(p.seed, n) + K_GROUP * (uint64_t)((e >> 2) + 1u);
+            OutT* out = reinterpret_cast<OutT*>(p.packed) + ((((uint64_t)plane * s.HW) + first[k]) >> 2);
+#pragma unroll
+            for (int r = 0; r < P2; ++r) {
+                if ((uint32_t)r < rows[k]) *out = (OutT)quant_row<Q>(vxy[k][r], vzw[k][r], stored2, delta2, scale2, rng_mix(ctr));
+                out += W4;
+                ctr += p.rng_row_step;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// general kernel: one CTA per plane, any shape
+// ------------------------------------------------------------------------------------------------
+template <typename XT, typename LT, int Q>
+__global__ void __launch_bounds__(256)
+pg_general_kernel(const XT* __restrict__ x, LT* lfc, uint32_t* packed, uint32_t* __restrict__ stats, Shape s,
+                  uint64_t seed) {
+    constexpr uint32_t PER = 32 / Q;
+    constexpr float qmax = (float)((1 << Q) - 1);
+    __shared__ uint32_t s_kmin, s_kmax;
+    __shared__ float s_delta, s_scale;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t plane = blockIdx.x;
+    const uint32_t n = plane / s.C, c = plane - n * s.C;
+    const XT* xp = x + (size_t)plane * s.HW;
+    LT* lp = lfc + (size_t)plane * s.TPP;
+    if (tid == 0) {
+        s_kmin = 0u;
+        s_kmax = 0u;
+    }
+    __syncthreads();
+    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+    for (uint32_t t = tid; t < s.TPP; t += 256u) {
+        float xmin, xmax;
+        const float mean = tile_mean(xp, s, t / s.Wb, t % s.Wb, xmin, xmax);
+        Elem<LT>::store(lp + t, mean);
+        const float stored = Elem<LT>::round(mean);
+        lo = fminf(lo, __fsub_rn(xmin, stored));
+        hi = fmaxf(hi, __fsub_rn(xmax, stored));
+    }
+    const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
+    const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+    if ((tid & 31u) == 0u) {
+        atomicMax(&s_kmin, kmin);
+        atomicMax(&s_kmax, kmax);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const PgQ q = pg_params(key_float(~s_kmin), key_float(s_kmax), Q);
+        s_delta = q.delta;
+        s_scale = q.scale;
+        stats[plane] = pg_stats_word(q);
+    }
+    __syncthreads();      // also makes this CTA's low-frequency values visible to all its threads
+    const float delta = s_delta, scale = s_scale;
+    const uint64_t base = rng_sample_base(seed, n);
+    const uint64_t i0 = (uint64_t)plane * s.HW, i1 = i0 + s.HW;       // the plane's global element range
+    const uint64_t w0 = i0 / PER, w1 = (i1 + PER - 1) / PER;
+    for (uint64_t word = w0 + tid; word < w1; word += 256u) {
+        const uint64_t a = max(word * PER, i0), b = min((word + 1) * PER, i1);
+        uint32_t acc = 0;
+        uint32_t cur_g = 0xFFFFFFFFu;
+        uint64_t z = 0;
+        for (uint64_t i = a; i < b; ++i) {
+            const uint32_t ep = (uint32_t)(i - i0);
+            const uint32_t h = ep / s.W, w = ep - h * s.W;
+            const uint32_t e = c * s.HW + ep;
+            if ((e >> 2) != cur_g) {
+                cur_g = e >> 2;
+                z = rng_group(base, cur_g);
+            }
+            const float l = Elem<LT>::load(lp + (h / s.B) * s.Wb + (w / s.B));
+            const float r = __fsub_rn(Elem<XT>::load(xp + ep), l);
+            const uint32_t field = (uint32_t)(z >> (16 * (e & 3))) & 0xFFFFu;
+            const uint32_t code = quant_bits(r, delta, scale, qmax, field) - MAGIC_CEIL_BITS;
+            acc |= code << ((uint32_t)(i - word * PER) * Q);
+        }
+        // a word shared with a neighbouring plane (or the zero-padded end of the stream) is merged into the
+        // pre-cleared buffer; every other word is written whole
+        if (b - a == PER) packed[word] = acc;
+        else atomicOr(packed + word, acc);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// decompress: x_hat = UpSampling(H^L) + (Delta_b * V^H + delta_b)   (Sec. 4.2, Eq. 10)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pg_unpack_stats(uint32_t w, float& delta, float& step) {
+    delta = __uint_as_float(w << 16);
+    step = __uint_as_float(w & 0xFFFF0000u);
+}
+
+// W % 4 == 0 and B a power of two >= 4: same tiling of the work as decompress_quad_kernel
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+pg_decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                          const uint32_t* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
+    constexpr uint32_t MASK = (1u << Q) - 1u;
+    const uint32_t n = blockIdx.y;
+    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
+    const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
+    const uint32_t* stats_n = stats + (size_t)n * d.C;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint32_t bits[QPT], sw[QPT];
+    float lf[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < d.qps) {
+            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
+            const uint32_t plane = fdiv(q, d.by_hwq);
+            const uint32_t rem = q - plane * d.hwq;
+            const uint32_t h = fdiv(rem, d.by_wq);
+            const uint32_t wq = rem - h * d.wq;
+            lf[k] = Elem<LT>::load(lfc_n + (size_t)plane * d.TPP + (h >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
+            sw[k] = __ldg(stats_n + plane);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < d.qps) {
+            float delta, step;
+            pg_unpack_stats(sw[k], delta, step);
+            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, reconstruct(bits[k] & MASK, step, delta, lf[k]),
+                            reconstruct((bits[k] >> Q) & MASK, step, delta, lf[k]),
+                            reconstruct((bits[k] >> (2 * Q)) & MASK, step, delta, lf[k]),
+                            reconstruct((bits[k] >> (3 * Q)) & MASK, step, delta, lf[k]));
+        }
+    }
+}
+
+// any shape: one thread per packed word
+template <typename XT, typename LT, int Q>
+__global__ void __launch_bounds__(256)
+pg_decompress_general_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                             const uint32_t* __restrict__ stats, XT* __restrict__ xhat, Shape s, uint64_t nwords) {
+    constexpr uint32_t PER = 32 / Q;
+    constexpr uint32_t MASK = (1u << Q) - 1u;
+    const uint64_t word = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (word >= nwords) return;
+    uint64_t i = word * PER;
+    uint64_t plane = i / s.HW;                       // global plane index n * C + c
+    uint32_t rem = (uint32_t)(i - plane * s.HW);
+    uint32_t h = rem / s.W, w = rem - h * s.W;
+    const uint32_t bits = packed[word];
+    uint64_t cur = ~0ull;
+    float delta = 0.f, step = 0.f;
+    for (uint32_t j = 0; j < PER && i < s.total; ++j, ++i) {
+        if (plane != cur) {
+            pg_unpack_stats(stats[plane], delta, step);
+            cur = plane;
+        }
+        const float l = Elem<LT>::load(lfc + plane * s.TPP + (h / s.B) * s.Wb + (w / s.B));
+        Elem<XT>::store(xhat + i, reconstruct((bits >> (j * Q)) & MASK, step, delta, l));
+        if (++w == s.W) {
+            w = 0;
+            if (++h == s.H) {
+                h = 0;
+                ++plane;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+struct PgPlan {
+    uint32_t spb, spp, G;
+    int32_t grid;
+};
+
+inline bool plan_pg_strip(const div_desc* d, const Shape& s, PgPlan* out) {
+    if (s.W % 4 != 0) return false;
+    if (!(s.B == 4 || s.B == 8) || s.P2 != s.B) return false;
+    if (!(d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return false;
+    const uint64_t planes = (uint64_t)s.N * s.C;
+    if (planes >= (1ull << 31)) return false;
+    PgPlan pl;
+    pl.spb = s.Wb * (s.P2 / 4);
+    const uint64_t spp = (uint64_t)s.Hb * pl.spb;
+    if (spp > PG_CAP) return false;
+    pl.spp = (uint32_t)spp;
+    uint64_t G = PG_CAP / pl.spp;
+    if (G > planes) G = planes;
+    pl.G = (uint32_t)G;
+    pl.grid = (int32_t)((planes + G - 1) / G);
+    *out = pl;
+    return true;
+}
+
+template <typename XT, typename LT>
+inline div_status launch_pg_strip(int qbits, uint32_t p2, const PgParams& prm, int grid, cudaStream_t st) {
+#define DIVK_PG_CASE(QQ, PP) \
+    if (qbits == QQ && p2 == PP) { pg_strip_kernel<XT, LT, QQ, PP><<<grid, PG_THREADS, 0, st>>>(prm); return DIV_OK; }
+    DIVK_PG_CASE(2, 8)
+    DIVK_PG_CASE(4, 8)
+    DIVK_PG_CASE(8, 8)
+    DIVK_PG_CASE(2, 4)
+    DIVK_PG_CASE(4, 4)
+    DIVK_PG_CASE(8, 4)
+#undef DIVK_PG_CASE
+    return DIV_ERR_PARAM;
+}
+
+inline div_status compress_pg_strip(const div_desc* d, const Shape& s, const div_layout& lo, const PgPlan& pl,
+                                    const void* x, uint8_t* blob, uint64_t seed, cudaStream_t st) {
+    PgParams prm;
+    prm.s = s;
+    prm.x = x;
+    prm.lfc = blob + lo.lfc_off;
+    prm.packed = blob + lo.packed_off;
+    prm.stats = reinterpret_cast<uint32_t*>(blob + lo.stats_off);
+    prm.seed = seed;
+    prm.rng_row_step = K_GROUP * (uint64_t)(s.W / 4u);
+    prm.planes = s.N * s.C;
+    prm.spb = pl.spb;
+    prm.spp = pl.spp;
+    prm.G = pl.G;
+    prm.tail_rows = s.H - (s.Hb - 1u) * s.B;
+    prm.by_spp = host_fastdiv(pl.spp);
+    prm.by_spb = host_fastdiv(pl.spb);
+    prm.by_c = host_fastdiv(s.C);
+    const uint32_t tail_cols = s.W - (s.Wb - 1u) * s.B;
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t rows = (i & 2) ? prm.tail_rows : s.B, cols = (i & 1) ? tail_cols : s.B;
+        const uint32_t cnt = rows * cols;
+        prm.cnt[i] = (float)cnt;
+        prm.inv_cnt[i] = (cnt & (cnt - 1)) == 0 ? 1.0f / (float)cnt : 0.f;      // exact for a power of two
+    }
+    typedef __nv_bfloat16 bf16;
+    div_status r;
+    if (d->x_dtype == DIV_F32)
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<float, float>(d->qbits, s.P2, prm, pl.grid, st)
+                                    : launch_pg_strip<float, bf16>(d->qbits, s.P2, prm, pl.grid, st);
+    else
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<bf16, float>(d->qbits, s.P2, prm, pl.grid, st)
+                                    : launch_pg_strip<bf16, bf16>(d->qbits, s.P2, prm, pl.grid, st);
+    if (r != DIV_OK) return r;
+    return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA;
+}
+
+}  // namespace divk

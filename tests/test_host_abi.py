@@ -50,6 +50,33 @@ def test_compressed_bytes_matches_closed_form(d):
     assert got.workspace_bytes >= 64 + 32 * n and got.workspace_bytes % 256 == 0
 
 
+@pytest.mark.parametrize("d", DESCS)
+def test_planegroup_bytes_matches_closed_form(d):
+    """Per-plane form: the same sections with 4 bytes of (delta, Delta) per plane and no scratch."""
+    n, c, h, w, b, q, xd, ld = d
+    got = binding.div_planegroup_bytes(binding.make_desc(*d))
+    ref = orc.plane_layout(n, c, h, w, b, q, xd, ld)
+    for field in ("lfc_off", "lfc_bytes", "packed_off", "packed_bytes", "stats_off", "stats_bytes",
+                  "total_bytes", "closed_form_bytes", "raw_bytes"):
+        assert getattr(got, field) == getattr(ref, field), field
+    assert got.workspace_bytes == 0 and got.stats_bytes == 4 * n * c
+
+
+def test_planegroup_refuses_too_many_planes_and_bad_flags():
+    L = binding.lib()
+    out = binding.DivLayout()
+    assert L.div_planegroup_bytes(ctypes.byref(binding.make_desc(2 ** 30, 2, 1, 1, 8, 2)), ctypes.byref(out)) == binding.DIV_ERR_SHAPE
+    assert L.div_planegroup_bytes(ctypes.byref(binding.make_desc(2 ** 30 - 1, 2, 1, 1, 8, 2)), ctypes.byref(out)) == binding.DIV_OK
+    assert L.div_planegroup_bytes(None, ctypes.byref(out)) == binding.DIV_ERR_NULL
+    d = binding.make_desc(2, 3, 8, 8, 8, 2)
+    assert L.div_planegroup_compress(ctypes.byref(d), None, None, 0, 0, None, 0) == binding.DIV_ERR_NULL
+    assert L.div_planegroup_compress(ctypes.byref(d), 16, 32, 0, 0, None, 4) == binding.DIV_ERR_PARAM
+    assert L.div_planegroup_compress(ctypes.byref(d), 16, 36, 1 << 20, 0, None, 0) == binding.DIV_ERR_ALIGN
+    assert L.div_planegroup_compress(ctypes.byref(d), 16, 32, 8, 0, None, 0) == binding.DIV_ERR_CAPACITY
+    assert L.div_planegroup_decompress(ctypes.byref(d), 16, 8, 32, None) == binding.DIV_ERR_CAPACITY
+    assert L.div_planegroup_decompress(ctypes.byref(d), 16, 1 << 20, 34, None) == binding.DIV_ERR_ALIGN
+
+
 def test_bad_descriptors_are_refused_on_the_host():
     L = binding.lib()
     out = binding.DivLayout()
