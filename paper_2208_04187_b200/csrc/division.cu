@@ -465,7 +465,7 @@ div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_p
     if (!(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_strip(desc, s, &pl)) {
         out->fused = 1;
         out->grid = pl.grid;
-        out->threads = PG_THREADS;
+        out->threads = (int32_t)pl.threads;
         out->chunk_elems = (int64_t)pl.G * s.HW;
         out->chunks_per_sample = (s.C + pl.G - 1) / pl.G;
     } else {

@@ -21,18 +21,17 @@
 
 namespace divk {
 
-#ifndef DIVK_PG_THREADS
-#define DIVK_PG_THREADS 256
+// Two shapes of the strip kernel: one strip slot per thread and up to PG1_THREADS threads (planes of up to
+// PG1_THREADS slots; more warps per SM), or two slots per thread and 256 threads (planes of up to 512 slots).
+#ifndef DIVK_PG1_THREADS
+#define DIVK_PG1_THREADS 448
 #endif
-#ifndef DIVK_PG_SLOTS
-#define DIVK_PG_SLOTS 2
-#endif
-#ifndef DIVK_PG_MIN_CTAS
-#define DIVK_PG_MIN_CTAS 2
-#endif
-constexpr int PG_THREADS = DIVK_PG_THREADS;
-constexpr int PG_K = DIVK_PG_SLOTS;               // strip slots a thread keeps in registers
-constexpr uint32_t PG_CAP = PG_THREADS * PG_K;    // strip slots of one CTA
+constexpr uint32_t PG1_THREADS = DIVK_PG1_THREADS;
+constexpr uint32_t PG2_THREADS = 256;
+constexpr uint32_t PG_CAP = 512;                  // most strip slots (and so most planes) of one CTA
+template <int K> struct PgShape;
+template <> struct PgShape<1> { static constexpr uint32_t MAX_THREADS = PG1_THREADS; };
+template <> struct PgShape<2> { static constexpr uint32_t MAX_THREADS = PG2_THREADS; };
 
 // ------------------------------------------------------------------------------------------------
 // the bfloat16 pair of one plane
@@ -98,8 +97,8 @@ struct PgParams {
     float cnt[4];
 };
 
-template <typename XT, typename LT, int Q, int P2>
-__global__ void __launch_bounds__(PG_THREADS, DIVK_PG_MIN_CTAS)
+template <typename XT, typename LT, int Q, int P2, int PG_K>
+__global__ void __launch_bounds__(PgShape<PG_K>::MAX_THREADS, 2)
 pg_strip_kernel(const PgParams p) {
     constexpr uint32_t LPT = P2 / 4;
     typedef typename PackedUnit<Q>::type OutT;
@@ -108,6 +107,7 @@ pg_strip_kernel(const PgParams p) {
 
     const Shape& s = p.s;
     const uint32_t tid = threadIdx.x;
+    const uint32_t PG_THREADS = blockDim.x;               // a multiple of 32
     const uint32_t row_bytes = s.W * (uint32_t)sizeof(XT);
     const uint32_t W4 = s.W >> 2;
     const uint32_t plane0 = blockIdx.x * p.G;
@@ -385,6 +385,7 @@ pg_decompress_general_kernel(const LT* __restrict__ lfc, const uint32_t* __restr
 // ------------------------------------------------------------------------------------------------
 struct PgPlan {
     uint32_t spb, spp, G;
+    uint32_t K, threads;
     int32_t grid;
 };
 
@@ -399,18 +400,25 @@ inline bool plan_pg_strip(const div_desc* d, const Shape& s, PgPlan* out) {
     const uint64_t spp = (uint64_t)s.Hb * pl.spb;
     if (spp > PG_CAP) return false;
     pl.spp = (uint32_t)spp;
-    uint64_t G = PG_CAP / pl.spp;
+    pl.K = spp <= PG1_THREADS ? 1u : 2u;
+    const uint32_t cap = pl.K == 1u ? PG1_THREADS : 2u * PG2_THREADS;
+    uint64_t G = cap / pl.spp;
     if (G > planes) G = planes;
     pl.G = (uint32_t)G;
+    pl.threads = pl.K == 1u ? ((pl.G * pl.spp + 31u) / 32u) * 32u : PG2_THREADS;
     pl.grid = (int32_t)((planes + G - 1) / G);
     *out = pl;
     return true;
 }
 
 template <typename XT, typename LT>
-inline div_status launch_pg_strip(int qbits, uint32_t p2, const PgParams& prm, int grid, cudaStream_t st) {
-#define DIVK_PG_CASE(QQ, PP) \
-    if (qbits == QQ && p2 == PP) { pg_strip_kernel<XT, LT, QQ, PP><<<grid, PG_THREADS, 0, st>>>(prm); return DIV_OK; }
+inline div_status launch_pg_strip(int qbits, uint32_t p2, const PgParams& prm, const PgPlan& pl, cudaStream_t st) {
+#define DIVK_PG_CASE(QQ, PP)                                                                        \
+    if (qbits == QQ && p2 == PP) {                                                                  \
+        if (pl.K == 1u) pg_strip_kernel<XT, LT, QQ, PP, 1><<<pl.grid, pl.threads, 0, st>>>(prm);    \
+        else pg_strip_kernel<XT, LT, QQ, PP, 2><<<pl.grid, pl.threads, 0, st>>>(prm);               \
+        return DIV_OK;                                                                              \
+    }
     DIVK_PG_CASE(2, 8)
     DIVK_PG_CASE(4, 8)
     DIVK_PG_CASE(8, 8)
@@ -449,11 +457,11 @@ inline div_status compress_pg_strip(const div_desc* d, const Shape& s, const div
     typedef __nv_bfloat16 bf16;
     div_status r;
     if (d->x_dtype == DIV_F32)
-        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<float, float>(d->qbits, s.P2, prm, pl.grid, st)
-                                    : launch_pg_strip<float, bf16>(d->qbits, s.P2, prm, pl.grid, st);
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<float, float>(d->qbits, s.P2, prm, pl, st)
+                                    : launch_pg_strip<float, bf16>(d->qbits, s.P2, prm, pl, st);
     else
-        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<bf16, float>(d->qbits, s.P2, prm, pl.grid, st)
-                                    : launch_pg_strip<bf16, bf16>(d->qbits, s.P2, prm, pl.grid, st);
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<bf16, float>(d->qbits, s.P2, prm, pl, st)
+                                    : launch_pg_strip<bf16, bf16>(d->qbits, s.P2, prm, pl, st);
     if (r != DIV_OK) return r;
     return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA;
 }
