@@ -225,7 +225,9 @@ div_status div_planegroup_compress(const div_desc* desc, const void* x_dev, void
                                    uint64_t seed, void* cuda_stream, uint32_t flags);
 div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev, size_t comp_bytes,
                                      void* xhat_dev, void* cuda_stream);
-/* plan.fused: 1 strip kernel, 0 general kernel; plan.decompress_fast: 1 quad kernel, 0 general. */
+/* plan.fused: 1 strip kernel, 2 small-plane kernel (tile row of at most 32 padded columns, B up to 16, Q in
+   {2,4,8}, sample size a multiple of 4), 0 general kernel; plan.decompress_fast: 1 quad kernel, 2 flat kernel
+   (total size a multiple of 4, planes up to 8192 elements), 0 general. */
 div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
 
 /* Which kernels a descriptor maps to on the current device.  desc, out: host. */

@@ -87,6 +87,9 @@ void make_layout_pg(const div_desc* d, const Shape& s, div_layout* out) {
     out->workspace_bytes = 0;
 }
 inline bool pg_shape_ok(const Shape& s) { return (uint64_t)s.N * s.C < (1ull << 31); }
+inline bool pg_decompress_flat_ok(const Shape& s) {
+    return (s.total % 4 == 0) && s.HW <= FLAT_MAX_HW && s.TPP <= 65535 && s.total / 4096 < 0x7FFFFFFFull;
+}
 
 FastDiv make_fastdiv(uint32_t d) {
     FastDiv f;
@@ -468,6 +471,13 @@ div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_p
         out->threads = (int32_t)pl.threads;
         out->chunk_elems = (int64_t)pl.G * s.HW;
         out->chunks_per_sample = (s.C + pl.G - 1) / pl.G;
+    } else if (PgSmall g; !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_small(desc, s, &g)) {
+        out->fused = 2;
+        out->grid = (int32_t)((g.planes + g.G - 1) / g.G);
+        out->threads = 256;
+        out->smem_bytes = (int32_t)pg_small_smem_bytes(g);
+        out->chunk_elems = (int64_t)g.G * s.HW;
+        out->chunks_per_sample = (s.C + g.G - 1) / g.G;
     } else {
         out->fused = 0;
         out->grid = (int32_t)(s.N * s.C);
@@ -475,7 +485,7 @@ div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_p
         out->chunk_elems = s.HW;
         out->chunks_per_sample = s.C;
     }
-    out->decompress_fast = decompress_fast_ok(s) ? 1 : 0;
+    out->decompress_fast = decompress_fast_ok(s) ? 1 : (pg_decompress_flat_ok(s) ? 2 : 0);
     return DIV_OK;
 }
 
@@ -493,9 +503,15 @@ div_status div_planegroup_compress(const div_desc* desc, const void* x_dev, void
     if (comp_capacity < lo.total_bytes) return DIV_ERR_CAPACITY;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     uint8_t* blob = (uint8_t*)comp_dev;
+    // kernels that store bytes or half-words leave the unused top of a partial last word alone: it is zero by contract
+    if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
+        cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
+        return DIV_ERR_CUDA;
     PgPlan pl;
     if (!(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_strip(desc, s, &pl))
         return compress_pg_strip(desc, s, lo, pl, x_dev, blob, seed, stream);
+    if (PgSmall g; !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_pg_small(desc, s, &g))
+        return compress_pg_small(desc, s, lo, g, x_dev, blob, seed, stream);
     // general kernel: words shared by two planes (and the zero-padded last word) are merged with atomic ORs
     // into a cleared buffer
     if (((uint64_t)s.HW * (uint64_t)desc->qbits) % 32u != 0 &&
@@ -550,6 +566,20 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
                 const uint32_t per_block = 256u * DEC_QPT;
                 dim3 grid((d.qps + per_block - 1) / per_block, s.N);
                 pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+            } else if (pg_decompress_flat_ok(s)) {
+                PgDecFlat d;
+                d.quads = s.total / 4;
+                d.HW = s.HW;
+                d.W = s.W;
+                d.Wb = s.Wb;
+                d.TPP = s.TPP;
+                d.table_words = flat_table_words(s.HW);
+                d.by_hw = make_fastdiv(s.HW);
+                d.by_w = make_fastdiv(s.W);
+                d.by_b = make_fastdiv(s.B);
+                const uint64_t g = (d.quads + 256u * DEC_QPT - 1) / (256u * DEC_QPT);
+                pg_decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<(unsigned)g, 256, 4u * d.table_words, stream>>>(
+                    lfc, packed, stats, (XT*)xhat_dev, d);
             } else {
                 const uint64_t g = (nwords + 255) / 256;
                 if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;

@@ -226,6 +226,158 @@ pg_strip_kernel(const PgParams p) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// small-plane kernel: planes of any width whose padded tile row fits a warp (the 14 x 14 and 7 x 7 maps).
+// A CTA takes G whole planes, contiguous in memory.  First half: a lane owns one tile column of one plane
+// (as in plane_stats_kernel): block means in the fixed order, stored low-frequency values (also kept in
+// shared memory), extremes per plane through shared-memory atomics.  Second half: one thread per 4
+// consecutive elements of the CTA's range (they may lie in different tiles, rows or planes; the tile of a
+// position comes from a table in shared memory); x is read a second time, from L1/L2.
+// ------------------------------------------------------------------------------------------------
+struct PgSmall {
+    Shape s;
+    const void* x;
+    void* lfc;
+    void* packed;
+    uint32_t* stats;
+    uint64_t seed;
+    uint32_t planes;            // N * C
+    uint32_t G;                 // planes per CTA; G * HW is a multiple of 4
+    uint32_t lanes_per_plane;   // Wb * P2
+    uint32_t planes_per_warp;   // 32 / lanes_per_plane
+    uint32_t table_words;       // 32-bit words of the tile table
+    FastDiv by_hw, by_w, by_b, by_c;
+};
+inline size_t pg_small_smem_bytes(const PgSmall& g) {
+    return 4ull * (g.table_words + (size_t)g.G * g.s.TPP + 4ull * g.G);
+}
+
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(256)
+pg_small_kernel(const PgSmall g) {
+    typedef typename PackedUnit<Q>::type OutT;
+    extern __shared__ uint32_t pg_smem[];
+    const Shape& s = g.s;
+    uint16_t* tile_of = reinterpret_cast<uint16_t*>(pg_smem);                 // position in a plane -> tile in the plane
+    float* lfc_s = reinterpret_cast<float*>(pg_smem + g.table_words);         // stored low-frequency values, G * TPP
+    uint32_t* s_key = pg_smem + g.table_words + g.G * s.TPP;                  // per plane: ~key(min), key(max)
+    float* s_par = reinterpret_cast<float*>(s_key + 2u * g.G);                // per plane: delta_b, 1 / Delta_b
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31u;
+    const uint32_t plane0 = blockIdx.x * g.G;
+    const uint32_t nplanes = min(g.G, g.planes - plane0);
+    const XT* x = reinterpret_cast<const XT*>(g.x);
+
+    for (uint32_t idx = tid; idx < s.HW; idx += 256u) {
+        const uint32_t h = fdiv(idx, g.by_w), w = idx - h * s.W;
+        tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * s.Wb + fdiv(w, g.by_b));
+    }
+    for (uint32_t i = tid; i < 2u * g.G; i += 256u) s_key[i] = 0u;
+    __syncthreads();
+
+    // ---- first half: lane = tile column
+    {
+        const uint32_t pl_local = lane / g.lanes_per_plane;
+        const uint32_t lw = lane - pl_local * g.lanes_per_plane;
+        const uint32_t bw = lw / P2, cw = lw % P2;
+        const uint32_t cols = (bw < s.Wb) ? min(s.B, s.W - bw * s.B) : 0u;
+        const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
+        const uint32_t col = bw * s.B + cw;
+        for (uint32_t pp = warp; pp * g.planes_per_warp < nplanes; pp += 8u) {
+            const uint32_t pc = pp * g.planes_per_warp + pl_local;          // plane inside the CTA
+            const bool ok = lane_ok && pc < nplanes;
+            const XT* xp = x + ((size_t)(plane0 + (ok ? pc : 0u)) * s.HW + (ok ? col : 0u));
+            LT* lp = reinterpret_cast<LT*>(g.lfc) + ((size_t)(plane0 + (ok ? pc : 0u)) * s.TPP + (ok ? bw : 0u));
+            float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+            for (uint32_t bh = 0; bh < s.Hb; ++bh) {
+                const uint32_t rows = min(s.B, s.H - bh * s.B);
+                float v[P2];
+#pragma unroll
+                for (int r = 0; r < P2; ++r)
+                    v[r] = (ok && (uint32_t)r < rows) ? Elem<XT>::load(xp + (size_t)(bh * s.B + r) * s.W) : 0.f;
+                float sum = tree8<P2>(v);
+#pragma unroll
+                for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+                float mean = 0.f;
+                if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));      // one lane per tile divides
+                mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
+                const float stored = Elem<LT>::round(mean);
+                if (ok) {
+                    if (cw == 0) {
+                        Elem<LT>::store(lp + (size_t)bh * s.Wb, mean);
+                        lfc_s[pc * s.TPP + bh * s.Wb + bw] = stored;
+                    }
+                    float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+#pragma unroll
+                    for (int r = 0; r < P2; ++r) {
+                        if ((uint32_t)r < rows) {
+                            blo = fminf(blo, v[r]);
+                            bhi = fmaxf(bhi, v[r]);
+                        }
+                    }
+                    // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
+                    lo = fminf(lo, __fsub_rn(blo, stored));
+                    hi = fmaxf(hi, __fsub_rn(bhi, stored));
+                }
+            }
+            // the columns of one tile meet through shuffles, the tiles of one plane in shared memory
+            uint32_t kmin = ~float_key(lo), kmax = float_key(hi);
+#pragma unroll
+            for (int m = 1; m < P2; m <<= 1) {
+                kmin = max(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, m));
+                kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, m));
+            }
+            if (pl_local < g.planes_per_warp && bw < s.Wb && cw == 0 && pc < nplanes) {
+                atomicMax(&s_key[2u * pc], kmin);
+                atomicMax(&s_key[2u * pc + 1u], kmax);
+            }
+        }
+    }
+    __syncthreads();
+    for (uint32_t i = tid; i < nplanes; i += 256u) {
+        const PgQ q = pg_params(key_float(~s_key[2u * i]), key_float(s_key[2u * i + 1u]), Q);
+        s_par[2u * i] = q.delta;
+        s_par[2u * i + 1u] = q.scale;
+        g.stats[plane0 + i] = pg_stats_word(q);
+    }
+    __syncthreads();
+
+    // ---- second half: Eq. 9 on 4 consecutive elements per step
+    {
+        constexpr float qmax = (float)((1 << Q) - 1);
+        const uint64_t e0 = (uint64_t)plane0 * s.HW;                      // first element of the CTA, a multiple of 4
+        const uint32_t nquads = (nplanes * s.HW) >> 2;
+        const XT* xc = x + e0;
+        OutT* out = reinterpret_cast<OutT*>(g.packed) + (e0 >> 2);
+        for (uint32_t qi = tid; qi < nquads; qi += 256u) {
+            uint64_t xy, zw;
+            StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(xc + (size_t)qi * 4u), xy, zw);
+            uint32_t pc = fdiv(qi * 4u, g.by_hw);
+            uint32_t rem = qi * 4u - pc * s.HW;
+            // the 4 elements lie in one sample (its size is a multiple of 4)
+            const uint32_t plane = plane0 + pc;
+            const uint32_t n = fdiv(plane, g.by_c);
+            const uint32_t e = (plane - n * s.C) * s.HW + rem;             // in-sample index of the first element
+            float lf[4], dl[4], sc[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                lf[i] = lfc_s[pc * s.TPP + tile_of[rem]];
+                dl[i] = s_par[2u * pc];
+                sc[i] = s_par[2u * pc + 1u];
+                if (++rem == s.HW) {
+                    rem = 0;
+                    ++pc;
+                }
+            }
+            const uint64_t z = rng_group(rng_sample_base(g.seed, n), e >> 2);
+            uint32_t b0, b1, b2, b3;
+            quant2(xy, pk2(lf[0], lf[1]), pk2(dl[0], dl[1]), pk2(sc[0], sc[1]), qmax, (uint32_t)z, b0, b1);
+            quant2(zw, pk2(lf[2], lf[3]), pk2(dl[2], dl[3]), pk2(sc[2], sc[3]), qmax, (uint32_t)(z >> 32), b2, b3);
+            constexpr uint32_t BIAS = QUANT2_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
+            out[qi] = (OutT)(b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // general kernel: one CTA per plane, any shape
 // ------------------------------------------------------------------------------------------------
 template <typename XT, typename LT, int Q>
@@ -380,6 +532,57 @@ pg_decompress_general_kernel(const LT* __restrict__ lfc, const uint32_t* __restr
     }
 }
 
+// total size a multiple of 4, planes of at most FLAT_MAX_HW elements, any W and B: one thread per 4 consecutive
+// elements of the flat stream; the tile of a position comes from a table in shared memory, the plane's pair
+// and low-frequency values from global memory (a few bytes per plane, served by L1)
+struct PgDecFlat {
+    uint64_t quads;          // N*C*H*W / 4
+    uint32_t HW, W, Wb, TPP;
+    uint32_t table_words;
+    FastDiv by_hw, by_w, by_b;
+};
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+pg_decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                          const uint32_t* __restrict__ stats, XT* __restrict__ xhat, PgDecFlat d) {
+    constexpr uint32_t MASK = (1u << Q) - 1u;
+    extern __shared__ uint32_t pg_smem[];
+    uint16_t* tile_of = reinterpret_cast<uint16_t*>(pg_smem);
+    for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
+        const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
+        tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
+    }
+    __syncthreads();
+    const uint64_t cta_e0 = (uint64_t)blockIdx.x * (1024u * QPT);           // first element of this CTA
+    const uint64_t cta_plane0 = cta_e0 / d.HW;
+    const uint32_t cta_rem0 = (uint32_t)(cta_e0 - cta_plane0 * d.HW);
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t lq = threadIdx.x + (uint32_t)k * 256u;               // quad inside the CTA
+        const uint64_t gq = (uint64_t)blockIdx.x * (256u * QPT) + lq;
+        if (gq < d.quads) {
+            const uint32_t bits = quad_bits<Q>(packed, gq);
+            const uint32_t loc = cta_rem0 + 4u * lq;                         // < HW + 4096 * QPT
+            const uint32_t dp = fdiv(loc, d.by_hw);
+            uint32_t rem = loc - dp * d.HW;
+            uint64_t plane = cta_plane0 + dp;
+            float v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                float delta, step;
+                pg_unpack_stats(__ldg(stats + plane), delta, step);
+                const float l = Elem<LT>::load(lfc + plane * d.TPP + tile_of[rem]);
+                v[i] = reconstruct((bits >> (i * Q)) & MASK, step, delta, l);
+                if (++rem == d.HW) {
+                    rem = 0;
+                    ++plane;
+                }
+            }
+            Quad<XT>::store(xhat + gq * 4u, v[0], v[1], v[2], v[3]);
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -462,6 +665,74 @@ inline div_status compress_pg_strip(const div_desc* d, const Shape& s, const div
     else
         r = d->lfc_dtype == DIV_F32 ? launch_pg_strip<bf16, float>(d->qbits, s.P2, prm, pl, st)
                                     : launch_pg_strip<bf16, bf16>(d->qbits, s.P2, prm, pl, st);
+    if (r != DIV_OK) return r;
+    return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA;
+}
+
+inline bool plan_pg_small(const div_desc* d, const Shape& s, PgSmall* out) {
+    if (!(d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return false;
+    if (!(s.P2 == 4 || s.P2 == 8 || s.P2 == 16)) return false;
+    if (s.Wb * s.P2 > 32u) return false;
+    if (s.CHW % 4 != 0 || s.HW > FLAT_MAX_HW) return false;
+    const uint64_t planes = (uint64_t)s.N * s.C;
+    if (planes >= (1ull << 31)) return false;
+    PgSmall g;
+    g.s = s;
+    g.planes = (uint32_t)planes;
+    g.lanes_per_plane = s.Wb * s.P2;
+    g.planes_per_warp = 32u / g.lanes_per_plane;
+    // planes per CTA: whole passes of the 8 warps (a multiple of 8, so G * HW is a multiple of 4), about 8192
+    // elements, bounded so that the per-plane arrays stay small
+    const uint32_t unit = 8u * g.planes_per_warp;
+    uint32_t m = 8192u / (unit * s.HW);
+    if (m < 1u) m = 1u;
+    while (m > 1u && (unit * m > 1024u || unit * m * s.TPP > 2048u)) --m;
+    g.G = unit * m;
+    if (g.G > 1024u || g.G * s.TPP > 4096u) return false;
+    g.table_words = flat_table_words(s.HW);
+    g.by_hw = host_fastdiv(s.HW);
+    g.by_w = host_fastdiv(s.W);
+    g.by_b = host_fastdiv(s.B);
+    g.by_c = host_fastdiv(s.C);
+    if (pg_small_smem_bytes(g) > 46000) return false;
+    *out = g;
+    return true;
+}
+
+template <typename XT, typename LT>
+inline div_status launch_pg_small(int qbits, uint32_t p2, const PgSmall& g, cudaStream_t st) {
+    const uint32_t grid = (g.planes + g.G - 1) / g.G;
+    const size_t smem = pg_small_smem_bytes(g);
+#define DIVK_PGS_CASE(QQ, PP) \
+    if (qbits == QQ && p2 == PP) { pg_small_kernel<XT, LT, QQ, PP><<<grid, 256, smem, st>>>(g); return DIV_OK; }
+    DIVK_PGS_CASE(2, 4)
+    DIVK_PGS_CASE(4, 4)
+    DIVK_PGS_CASE(8, 4)
+    DIVK_PGS_CASE(2, 8)
+    DIVK_PGS_CASE(4, 8)
+    DIVK_PGS_CASE(8, 8)
+    DIVK_PGS_CASE(2, 16)
+    DIVK_PGS_CASE(4, 16)
+    DIVK_PGS_CASE(8, 16)
+#undef DIVK_PGS_CASE
+    return DIV_ERR_PARAM;
+}
+
+inline div_status compress_pg_small(const div_desc* d, const Shape& s, const div_layout& lo, PgSmall g,
+                                    const void* x, uint8_t* blob, uint64_t seed, cudaStream_t st) {
+    g.x = x;
+    g.lfc = blob + lo.lfc_off;
+    g.packed = blob + lo.packed_off;
+    g.stats = reinterpret_cast<uint32_t*>(blob + lo.stats_off);
+    g.seed = seed;
+    typedef __nv_bfloat16 bf16;
+    div_status r;
+    if (d->x_dtype == DIV_F32)
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_small<float, float>(d->qbits, s.P2, g, st)
+                                    : launch_pg_small<float, bf16>(d->qbits, s.P2, g, st);
+    else
+        r = d->lfc_dtype == DIV_F32 ? launch_pg_small<bf16, float>(d->qbits, s.P2, g, st)
+                                    : launch_pg_small<bf16, bf16>(d->qbits, s.P2, g, st);
     if (r != DIV_OK) return r;
     return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA;
 }

@@ -70,12 +70,20 @@ STRIP = [
     ((2, 7, 28, 28), 8, 4, "f32", "bf16"), ((2, 3, 20, 12), 8, 8, "f32", "f32"), ((3, 4, 13, 20), 4, 2, "bf16", "bf16"),
     ((2, 600, 4, 4), 4, 2, "f32", "f32"), ((1, 1, 8, 8), 8, 2, "f32", "f32"), ((2, 9, 30, 36), 8, 4, "bf16", "f32"),
     ((1, 3, 128, 128), 8, 2, "f32", "f32"), ((5, 11, 8, 24), 4, 8, "f32", "bf16"), ((2, 130, 8, 8), 8, 2, "f32", "f32"),
+    ((1, 3, 1, 4), 4, 2, "f32", "f32"),          # 12 elements: the last packed word is partial
 ]
-# shapes only the general kernel takes (odd widths, other block sizes, Q = 1, planes that share packed words)
+# shapes the small-plane kernel takes: any width, padded tile row of at most 32 columns, sample size a multiple of 4
+SMALL_PLANE = [
+    ((2, 8, 14, 14), 8, 2, "f32", "f32"), ((3, 16, 7, 7), 8, 2, "f32", "f32"), ((2, 4, 9, 13), 4, 4, "f32", "f32"),
+    ((2, 40, 7, 7), 8, 4, "bf16", "bf16"), ((1, 4, 6, 10), 3, 2, "bf16", "f32"), ((2, 3, 12, 20), 12, 2, "f32", "bf16"),
+    ((130, 12, 14, 14), 8, 8, "f32", "f32"), ((5, 100, 7, 7), 8, 2, "f32", "bf16"), ((2, 6, 30, 30), 16, 2, "f32", "f32"),
+    ((3, 700, 2, 6), 4, 2, "f32", "f32"),
+]
+# shapes only the general kernel takes (sample size not a multiple of 4, other block sizes, Q = 1, wide odd planes)
 GENERAL_ONLY = [
-    ((2, 3, 14, 14), 8, 2, "f32", "f32"), ((2, 5, 7, 7), 8, 2, "f32", "f32"), ((2, 3, 9, 13), 4, 4, "f32", "f32"),
-    ((1, 4, 16, 16), 8, 1, "f32", "f32"), ((2, 3, 12, 20), 12, 2, "f32", "bf16"), ((3, 3, 5, 5), 16, 8, "bf16", "bf16"),
-    ((1, 2, 160, 160), 8, 2, "f32", "f32"), ((2, 2, 3, 1), 2, 1, "f32", "f32"), ((1, 7, 6, 10), 3, 2, "bf16", "f32"),
+    ((2, 3, 7, 7), 8, 2, "f32", "f32"), ((2, 5, 7, 7), 8, 2, "f32", "f32"), ((2, 3, 9, 13), 4, 4, "f32", "f32"),
+    ((1, 4, 16, 16), 8, 1, "f32", "f32"), ((2, 3, 13, 50), 8, 2, "f32", "bf16"), ((3, 3, 5, 5), 16, 8, "bf16", "bf16"),
+    ((1, 2, 160, 160), 8, 2, "f32", "f32"), ((2, 2, 3, 1), 2, 1, "f32", "f32"), ((1, 8, 6, 10), 64, 1, "bf16", "f32"),
 ]
 
 
@@ -85,13 +93,20 @@ def test_strip_kernel_matches_the_checker(shape, block, q, xd, ld, kind):
     assert_parity(make_input(shape, kind, 31, xd), block, q, 77, xd, ld, expect_fused=1)
 
 
-@pytest.mark.parametrize("shape,block,q,xd,ld", STRIP + GENERAL_ONLY)
+@pytest.mark.parametrize("shape,block,q,xd,ld", SMALL_PLANE)
+@pytest.mark.parametrize("kind", ["bn", "relu"])
+def test_small_plane_kernel_matches_the_checker(shape, block, q, xd, ld, kind):
+    codec = assert_parity(make_input(shape, kind, 34, xd), block, q, 80, xd, ld, expect_fused=2)
+    assert codec.plan().decompress_fast == 2
+
+
+@pytest.mark.parametrize("shape,block,q,xd,ld", STRIP + SMALL_PLANE + GENERAL_ONLY)
 def test_general_kernel_matches_the_checker(shape, block, q, xd, ld):
     assert_parity(make_input(shape, "bn", 32, xd), block, q, 78, xd, ld, flags=GENERAL, expect_fused=0)
 
 
 @pytest.mark.parametrize("shape,block,q,xd,ld", GENERAL_ONLY)
-def test_default_path_on_shapes_outside_the_strip_kernel(shape, block, q, xd, ld):
+def test_default_path_on_shapes_outside_the_special_kernels(shape, block, q, xd, ld):
     assert_parity(make_input(shape, "relu", 33, xd), block, q, 79, xd, ld, expect_fused=0)
 
 
@@ -106,6 +121,11 @@ def test_degenerate_planes_store_a_zero_step():
         got = orc.parse_plane_blob(codec.blob.cpu().numpy(), 2, 4, 16, 16, 8, 2)
         assert got.step[0, 1] == 0 and got.step[1, 2] == 0 and got.step[1, 3] == 0
         assert not got.codes[0, 1].any() and not got.codes[1, 2].any()
+    # the same on planes of the small-plane kernel
+    y = synth.activation_map(2, 4, 14, 14, "bn", 5)
+    y[0, 1] = 0.0
+    y[1, 2] = 3.25
+    assert_parity(y, 8, 2, 5, expect_fused=2)
 
 
 def test_extreme_magnitudes():
@@ -117,6 +137,7 @@ def test_extreme_magnitudes():
     x[1, 1, 0, 1] = -1.5e38    # range close to the largest fp32 number, reciprocal of the step subnormal
     for flags in (0, GENERAL):
         assert_parity(x, 8, 2, 9, flags=flags)
+    assert_parity(x[:, :2, :14, :14].copy(), 8, 2, 9, expect_fused=2)
 
 
 def test_outputs_do_not_depend_on_the_kernel():
