@@ -37,6 +37,12 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_TRAFFIC_BYTES = 214477824      # 206767872 read + 7709952 written (profiles/lagged_kernel_and_decompress_quad_map_64x64x112x112.md)
 
 
+# The same for the per-plane strip kernel on that map: one ncu capture on 40 of the 64 samples (128.47 MB read +
+# 7.12 MB written for 128.45 MB of x), scaled by 64/40 -- the kernel's traffic is proportional to the planes it
+# processes (profiles/pg_strip_kernel_map_40x64x112x112.md).
+PG_NCU_TRAFFIC_BYTES = int((128467200 + 7116032) * 64 / 40)
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -273,6 +279,66 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
+    # ---- the per-plane form (one bfloat16 (delta, Delta) pair per plane): same maps, same order, own timed loop ----
+    plane_groups = None
+    if not args.no_plane_groups:
+        pg = [binding.PlaneGroupCodec(*s.shape, s.block, s.qbits, s.x_dtype, s.lfc_dtype, device=device) for s in specs]
+        pg_plans = [c.plan() for c in pg]
+        pg_steps = max(3, min(args.steps, 100))
+
+        def pg_step(record=None):
+            for i, c in enumerate(pg):
+                if record is not None:
+                    record[0][i][0].record()
+                c.compress(dev_x[i], seed=0)
+                if record is not None:
+                    record[0][i][1].record()
+            for i, c in enumerate(pg):
+                if record is not None:
+                    record[1][i][0].record()
+                c.decompress(out=dev_out[i])
+                if record is not None:
+                    record[1][i][1].record()
+
+        for _ in range(3):
+            pg_step()
+        barrier()
+        pg_rec = [[[(ev(), ev()) for _ in pg] for _ in range(2)] for _ in range(pg_steps)]
+        p0, p1 = ev(), ev()
+        p0.record()
+        for k in range(pg_steps):
+            pg_step(pg_rec[k])
+        p1.record()
+        barrier()
+        pg_ms = p0.elapsed_time(p1) / pg_steps
+        pg_comp = [statistics.mean(pg_rec[k][0][i][0].elapsed_time(pg_rec[k][0][i][1]) for k in range(pg_steps))
+                   for i in range(len(pg))]
+        pg_dec = [statistics.mean(pg_rec[k][1][i][0].elapsed_time(pg_rec[k][1][i][1]) for k in range(pg_steps))
+                  for i in range(len(pg))]
+        pg_names = {1: "pg_strip_kernel", 2: "pg_small_kernel", 0: "pg_general_kernel"}
+        pg_dec_names = {1: "pg_decompress_quad_kernel", 2: "pg_decompress_flat_kernel", 0: "pg_decompress_general_kernel"}
+        pg_algo = [int(c.layout.raw_bytes) + int(c.layout.closed_form_bytes) for c in pg]
+        pg_dom = max(range(len(pg)), key=lambda i: pg_comp[i])
+        pg_peak, pg_peak_kind = measured_peak()
+        pg_dom_gbs = pg_algo[pg_dom] / (pg_comp[pg_dom] * 1e-3) / 1e9
+        plane_groups = {
+            "what": "the same step with one bfloat16 (delta, Delta) pair per (sample, channel) plane "
+                    "(div_planegroup_compress / div_planegroup_decompress), this rank",
+            "value": raw_bytes / (pg_ms * 1e-3) / 1e9, "unit": UNIT, "steps": pg_steps, "ms_per_step": pg_ms,
+            "compression_ratio": raw_bytes / sum(int(c.layout.closed_form_bytes) for c in pg),
+            "gpu_launches": 2 * len(pg) * pg_steps,
+            "per_map": [{"map": "x".join(map(str, s.shape)), "compress_kernel": pg_names[int(p.fused)],
+                         "decompress_kernel": pg_dec_names[int(p.decompress_fast)],
+                         "compress_us": round(cm * 1e3, 2), "compress_GBps": round(b / cm / 1e6, 1),
+                         "decompress_us": round(dm * 1e3, 2), "decompress_GBps": round(b / dm / 1e6, 1)}
+                        for s, p, cm, dm, b in zip(specs, pg_plans, pg_comp, pg_dec, pg_algo)],
+            "roofline": {"bound": "hbm", "kernel": pg_names[int(pg_plans[pg_dom].fused)] + " on " +
+                         "x".join(map(str, specs[pg_dom].shape)), "achieved": pg_dom_gbs, "peak": pg_peak,
+                         "unit": "GB/s", "frac": pg_dom_gbs / pg_peak, "peak_kind": f"of {pg_peak_kind}",
+                         "traffic": PG_NCU_TRAFFIC_BYTES if specs[pg_dom].shape == (64, 64, 112, 112) else None,
+                         "algorithmic_bytes_per_launch": pg_algo[pg_dom]},
+        }
+
     ms_per_step = total_ms / args.steps
     job_ms, job_bytes = aggregate_over_ranks(ms_per_step, float(raw_bytes), dist if world > 1 else None, device)
     e2e_job_ms, _ = aggregate_over_ranks(e2e_ms, float(raw_bytes), dist if world > 1 else None, device)
@@ -321,6 +387,7 @@ def run_ours(args):
         "roofline_all_decompress": {"bound": "hbm", "kernel": "all decompress calls of the step", "achieved": dec_gbs,
                                     "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": f"of {peak_kind}"},
         "cpu_baseline": cpu,
+        "plane_groups": plane_groups,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
                 "steps": e2e_steps},
@@ -339,6 +406,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-plane-groups", action="store_true", help="skip the extra timed loop of the per-plane form")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
     ap.add_argument("--compress-flags", type=int, default=0,
                     help="DIV_FLAG_* bits passed to div_compress_ex (profiling aid: 4 = strip ring kernel instead of the lagged one)")
