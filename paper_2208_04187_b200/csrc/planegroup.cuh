@@ -21,20 +21,14 @@
 
 namespace divk {
 
-// Two shapes of the strip kernel: one strip slot per thread and up to PG1_THREADS threads (planes of up to
-// PG1_THREADS slots; more warps per SM), or two slots per thread and 256 threads (planes of up to 512 slots).
-#ifndef DIVK_PG1_THREADS
-#define DIVK_PG1_THREADS 448
-#endif
+// Shape of the strip kernel: one strip slot per thread; a CTA of up to PG_MAX_THREADS threads takes one large
+// plane, or a few whole small planes (CTAs of about DIVK_PG_SMALL_CTA threads, twice that for medium planes).
 #ifndef DIVK_PG_SMALL_CTA
 #define DIVK_PG_SMALL_CTA 128
 #endif
-constexpr uint32_t PG1_THREADS = DIVK_PG1_THREADS;
-constexpr uint32_t PG2_THREADS = 256;
-constexpr uint32_t PG_CAP = 512;                  // most strip slots (and so most planes) of one CTA
-template <int K> struct PgShape;
-template <> struct PgShape<1> { static constexpr uint32_t MAX_THREADS = PG1_THREADS; };
-template <> struct PgShape<2> { static constexpr uint32_t MAX_THREADS = PG2_THREADS; };
+constexpr uint32_t PG_MAX_THREADS = 512;
+constexpr int PG_K = 1;                           // strip slots a thread keeps in registers
+constexpr uint32_t PG_CAP = PG_MAX_THREADS;       // most strip slots of a plane
 
 // ------------------------------------------------------------------------------------------------
 // the bfloat16 pair of one plane
@@ -100,13 +94,13 @@ struct PgParams {
     float cnt[4];
 };
 
-template <typename XT, typename LT, int Q, int P2, int PG_K>
-__global__ void __launch_bounds__(PgShape<PG_K>::MAX_THREADS, 2)
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(PG_MAX_THREADS, 2)
 pg_strip_kernel(const PgParams p) {
     constexpr uint32_t LPT = P2 / 4;
     typedef typename PackedUnit<Q>::type OutT;
-    __shared__ uint32_t s_key[2 * PG_CAP];     // per plane of this CTA: ~key(min), key(max)
-    __shared__ float s_par[2 * PG_CAP];        // per plane: delta_b, 1 / Delta_b
+    __shared__ uint32_t s_key[2 * PG_MAX_THREADS];     // per plane of this CTA: ~key(min), key(max)
+    __shared__ float s_par[2 * PG_MAX_THREADS];        // per plane: delta_b, 1 / Delta_b
 
     const Shape& s = p.s;
     const uint32_t tid = threadIdx.x;
@@ -591,7 +585,7 @@ pg_decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict
 // ------------------------------------------------------------------------------------------------
 struct PgPlan {
     uint32_t spb, spp, G;
-    uint32_t K, threads;
+    uint32_t threads;
     int32_t grid;
 };
 
@@ -601,22 +595,23 @@ inline bool plan_pg_strip(const div_desc* d, const Shape& s, PgPlan* out) {
     if (!(d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return false;
     const uint64_t planes = (uint64_t)s.N * s.C;
     if (planes >= (1ull << 31)) return false;
-    PgPlan pl;
+    PgPlan pl = PgPlan();
     pl.spb = s.Wb * (s.P2 / 4);
     const uint64_t spp = (uint64_t)s.Hb * pl.spb;
     if (spp > PG_CAP) return false;
     pl.spp = (uint32_t)spp;
-    pl.K = spp <= PG1_THREADS ? 1u : 2u;
-    // small planes: CTAs of about DIVK_PG_SMALL_CTA threads (twice that for medium ones), so that several CTAs
-    // share an SM and their load and compute phases interleave (measured: 56 x 56 planes 64 -> 56 us,
-    // 28 x 28 planes 41 -> 33 us on the 64-sample ResNet-50 maps)
-    uint32_t cap = pl.K == 1u ? PG1_THREADS : 2u * PG2_THREADS;
-    if (pl.K == 1u && pl.spp <= DIVK_PG_SMALL_CTA / 2u) cap = DIVK_PG_SMALL_CTA;
-    else if (pl.K == 1u && pl.spp <= 2u * DIVK_PG_SMALL_CTA) cap = 2u * DIVK_PG_SMALL_CTA;
+    // CTAs of about DIVK_PG_SMALL_CTA threads (twice that for medium planes), so that several CTAs share an SM
+    // and their load and compute phases interleave (measured on the 64-sample ResNet-50 maps: 56 x 56 planes
+    // 64 -> 56 us, 28 x 28 planes 41 -> 33 us).  A larger plane takes one CTA of its own; splitting it over a
+    // thread-block cluster of 2 or 4 smaller CTAs that exchange their extremes through distributed shared
+    // memory was measured slower (70 and 78 us against 66 us on the 112 x 112 planes).
+    uint32_t cap = PG_MAX_THREADS;
+    if (pl.spp <= DIVK_PG_SMALL_CTA / 2u) cap = DIVK_PG_SMALL_CTA;
+    else if (pl.spp <= 2u * DIVK_PG_SMALL_CTA) cap = 2u * DIVK_PG_SMALL_CTA;
     uint64_t G = cap / pl.spp;
     if (G > planes) G = planes;
     pl.G = (uint32_t)G;
-    pl.threads = pl.K == 1u ? ((pl.G * pl.spp + 31u) / 32u) * 32u : PG2_THREADS;
+    pl.threads = ((pl.G * pl.spp + 31u) / 32u) * 32u;
     pl.grid = (int32_t)((planes + G - 1) / G);
     *out = pl;
     return true;
@@ -624,12 +619,8 @@ inline bool plan_pg_strip(const div_desc* d, const Shape& s, PgPlan* out) {
 
 template <typename XT, typename LT>
 inline div_status launch_pg_strip(int qbits, uint32_t p2, const PgParams& prm, const PgPlan& pl, cudaStream_t st) {
-#define DIVK_PG_CASE(QQ, PP)                                                                        \
-    if (qbits == QQ && p2 == PP) {                                                                  \
-        if (pl.K == 1u) pg_strip_kernel<XT, LT, QQ, PP, 1><<<pl.grid, pl.threads, 0, st>>>(prm);    \
-        else pg_strip_kernel<XT, LT, QQ, PP, 2><<<pl.grid, pl.threads, 0, st>>>(prm);               \
-        return DIV_OK;                                                                              \
-    }
+#define DIVK_PG_CASE(QQ, PP) \
+    if (qbits == QQ && p2 == PP) { pg_strip_kernel<XT, LT, QQ, PP><<<pl.grid, pl.threads, 0, st>>>(prm); return DIV_OK; }
     DIVK_PG_CASE(2, 8)
     DIVK_PG_CASE(4, 8)
     DIVK_PG_CASE(8, 8)
