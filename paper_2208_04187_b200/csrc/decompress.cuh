@@ -51,18 +51,23 @@ decompress_general_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict
 }
 
 // ---------------------------------------------------------------------------------------------
-// vector kernel: W % 4 == 0, B a power of two >= 4 (so that 4 consecutive elements share a tile).
-// One thread produces QPT quads (4 elements each, one 16-byte or 8-byte store); quads of a warp are
-// consecutive, so every store instruction of a warp writes one contiguous 512-byte (fp32) span.
-// grid = (ceil(quads_per_sample / (256*QPT)), N)
+// vector kernel: W % 4 == 0, B a power of two >= 4 (so that 4 consecutive elements share a tile, and so do
+// the 4 rows of an aligned row group).  One thread produces 4 quads (4 elements each, one 16-byte or 8-byte
+// store): the same 4 columns of 4 consecutive rows, which share one low-frequency value and one set of index
+// arithmetic.  Threads of a warp take consecutive quads of a row group, so every store instruction of a warp
+// writes contiguous spans.
+// grid = (ceil(C * ceil(H/4) * (W/4) / 256), N)
 // ---------------------------------------------------------------------------------------------
 struct DecFast {
     uint32_t qps;        // quads per sample = CHW / 4
     uint32_t C, TPP, Wb;
     uint32_t log2B;
-    FastDiv by_hwq;      // / (HW/4)
+    uint32_t H;
+    uint32_t hwq, wq;    // quads per plane and per row
+    uint32_t ipp;        // work items per plane = ceil(H/4) * (W/4)
+    uint32_t items;      // work items per sample = C * ipp
+    FastDiv by_ipp;      // / ipp
     FastDiv by_wq;       // / (W/4)
-    uint32_t hwq, wq;
 };
 
 template <typename XT> struct Quad;
@@ -143,35 +148,31 @@ template <typename XT, typename LT, int Q, int QPT>
 __global__ void __launch_bounds__(256)
 decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
+    static_assert(QPT == 4, "a work item is 4 rows high");
     __shared__ DeqTable<Q> table;
     const uint32_t n = blockIdx.y;
     table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
     __syncthreads();
-    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
-    const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
-    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
-
-    uint32_t bits[QPT];
-    float lf[QPT];
+    const uint32_t item = blockIdx.x * 256u + threadIdx.x;
+    if (item >= d.items) return;
+    const uint32_t plane = fdiv(item, d.by_ipp);
+    const uint32_t rem = item - plane * d.ipp;
+    const uint32_t hq = fdiv(rem, d.by_wq);
+    const uint32_t wq = rem - hq * d.wq;
+    const uint32_t h0 = hq * 4u;
+    const float lf = Elem<LT>::load(lfc + ((size_t)n * d.C + plane) * d.TPP + (h0 >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
+    const uint64_t quad0 = (uint64_t)n * d.qps + plane * d.hwq + h0 * d.wq + wq;      // first row's quad
+    const uint32_t rows = min(4u, d.H - h0);
+    uint32_t bits[4];
 #pragma unroll
-    for (int k = 0; k < QPT; ++k) {
-        const uint32_t q = q0 + k * 256u;
-        if (q < d.qps) {
-            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
-            const uint32_t plane = fdiv(q, d.by_hwq);
-            const uint32_t rem = q - plane * d.hwq;
-            const uint32_t h = fdiv(rem, d.by_wq);
-            const uint32_t wq = rem - h * d.wq;
-            lf[k] = Elem<LT>::load(lfc_n + (size_t)plane * d.TPP + (h >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
-        }
-    }
+    for (int r = 0; r < 4; ++r)
+        if ((uint32_t)r < rows) bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * d.wq);
 #pragma unroll
-    for (int k = 0; k < QPT; ++k) {
-        const uint32_t q = q0 + k * 256u;
-        if (q < d.qps) {
-            const float4 hq = table.quad(bits[k]);
-            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, __fadd_rn(lf[k], hq.x), __fadd_rn(lf[k], hq.y),
-                            __fadd_rn(lf[k], hq.z), __fadd_rn(lf[k], hq.w));
+    for (int r = 0; r < 4; ++r) {
+        if ((uint32_t)r < rows) {
+            const float4 hq4 = table.quad(bits[r]);
+            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * d.wq) * 4u, __fadd_rn(lf, hq4.x), __fadd_rn(lf, hq4.y),
+                            __fadd_rn(lf, hq4.z), __fadd_rn(lf, hq4.w));
         }
     }
 }

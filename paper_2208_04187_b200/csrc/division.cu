@@ -353,12 +353,14 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 d.Wb = s.Wb;
                 d.log2B = 0;
                 while ((1u << d.log2B) < s.B) ++d.log2B;
+                d.H = s.H;
                 d.hwq = s.HW / 4;
                 d.wq = s.W / 4;
-                d.by_hwq = make_fastdiv(d.hwq);
+                d.ipp = ((s.H + 3u) / 4u) * d.wq;
+                d.items = s.C * d.ipp;
+                d.by_ipp = make_fastdiv(d.ipp);
                 d.by_wq = make_fastdiv(d.wq);
-                const uint32_t per_block = 256u * DEC_QPT;
-                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                dim3 grid((d.items + 255u) / 256u, s.N);
                 decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
             } else if (decompress_flat_ok(s)) {
                 DecFlat d;
@@ -559,12 +561,14 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
                 d.Wb = s.Wb;
                 d.log2B = 0;
                 while ((1u << d.log2B) < s.B) ++d.log2B;
+                d.H = s.H;
                 d.hwq = s.HW / 4;
                 d.wq = s.W / 4;
-                d.by_hwq = make_fastdiv(d.hwq);
+                d.ipp = ((s.H + 3u) / 4u) * d.wq;
+                d.items = s.C * d.ipp;
+                d.by_ipp = make_fastdiv(d.ipp);
                 d.by_wq = make_fastdiv(d.wq);
-                const uint32_t per_block = 256u * DEC_QPT;
-                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                dim3 grid((d.items + 255u) / 256u, s.N);
                 pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
             } else if (pg_decompress_flat_ok(s)) {
                 PgDecFlat d;

@@ -456,42 +456,39 @@ __device__ __forceinline__ void pg_unpack_stats(uint32_t w, float& delta, float&
     step = __uint_as_float(w & 0xFFFF0000u);
 }
 
-// W % 4 == 0 and B a power of two >= 4: same tiling of the work as decompress_quad_kernel
+// W % 4 == 0 and B a power of two >= 4: same tiling of the work as decompress_quad_kernel (a thread produces
+// the same 4 columns of 4 consecutive rows: one low-frequency value, one plane pair, one set of index arithmetic)
 template <typename XT, typename LT, int Q, int QPT>
 __global__ void __launch_bounds__(256)
 pg_decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                           const uint32_t* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
+    static_assert(QPT == 4, "a work item is 4 rows high");
     constexpr uint32_t MASK = (1u << Q) - 1u;
     const uint32_t n = blockIdx.y;
-    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
-    const LT* lfc_n = lfc + (size_t)n * d.C * d.TPP;
-    const uint32_t* stats_n = stats + (size_t)n * d.C;
-    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
-    uint32_t bits[QPT], sw[QPT];
-    float lf[QPT];
+    const uint32_t item = blockIdx.x * 256u + threadIdx.x;
+    if (item >= d.items) return;
+    const uint32_t plane = fdiv(item, d.by_ipp);
+    const uint32_t rem = item - plane * d.ipp;
+    const uint32_t hq = fdiv(rem, d.by_wq);
+    const uint32_t wq = rem - hq * d.wq;
+    const uint32_t h0 = hq * 4u;
+    const size_t gp = (size_t)n * d.C + plane;
+    const float lf = Elem<LT>::load(lfc + gp * d.TPP + (h0 >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
+    float delta, step;
+    pg_unpack_stats(__ldg(stats + gp), delta, step);
+    const uint64_t quad0 = (uint64_t)n * d.qps + plane * d.hwq + h0 * d.wq + wq;
+    const uint32_t rows = min(4u, d.H - h0);
+    uint32_t bits[4];
 #pragma unroll
-    for (int k = 0; k < QPT; ++k) {
-        const uint32_t q = q0 + k * 256u;
-        if (q < d.qps) {
-            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
-            const uint32_t plane = fdiv(q, d.by_hwq);
-            const uint32_t rem = q - plane * d.hwq;
-            const uint32_t h = fdiv(rem, d.by_wq);
-            const uint32_t wq = rem - h * d.wq;
-            lf[k] = Elem<LT>::load(lfc_n + (size_t)plane * d.TPP + (h >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
-            sw[k] = __ldg(stats_n + plane);
-        }
-    }
+    for (int r = 0; r < 4; ++r)
+        if ((uint32_t)r < rows) bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * d.wq);
 #pragma unroll
-    for (int k = 0; k < QPT; ++k) {
-        const uint32_t q = q0 + k * 256u;
-        if (q < d.qps) {
-            float delta, step;
-            pg_unpack_stats(sw[k], delta, step);
-            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, reconstruct(bits[k] & MASK, step, delta, lf[k]),
-                            reconstruct((bits[k] >> Q) & MASK, step, delta, lf[k]),
-                            reconstruct((bits[k] >> (2 * Q)) & MASK, step, delta, lf[k]),
-                            reconstruct((bits[k] >> (3 * Q)) & MASK, step, delta, lf[k]));
+    for (int r = 0; r < 4; ++r) {
+        if ((uint32_t)r < rows) {
+            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * d.wq) * 4u, reconstruct(bits[r] & MASK, step, delta, lf),
+                            reconstruct((bits[r] >> Q) & MASK, step, delta, lf),
+                            reconstruct((bits[r] >> (2 * Q)) & MASK, step, delta, lf),
+                            reconstruct((bits[r] >> (3 * Q)) & MASK, step, delta, lf));
         }
     }
 }
