@@ -537,3 +537,56 @@ def parse_plane_blob(blob: np.ndarray, n: int, c: int, h: int, w: int, block: in
     codes = unpack_codes(words, qbits, n * c * h * w).reshape(n, c, h * w)
     return PlaneCompressed((n, c, h, w), block, qbits, x_dtype, lfc_dtype, lfc, codes, words,
                            bf16_bits_to_f32(pair[:, :, 0].copy()), bf16_bits_to_f32(pair[:, :, 1].copy()), lo)
+
+
+# ----------------------------------------------------------------------------------------
+# ReLU and dropout operators with a packed 1-bit mask (the paper's appendix algorithms
+# "Relu operator" and "Dropout operator"; 1 bit per element in the byte count of Theorem 3A)
+# ----------------------------------------------------------------------------------------
+# Forward:  V = mask, H_out = V (.) H_in, V packed and cached.   Backward:  grad_in = V (.) grad_out.
+# Readings:
+#   * ReLU: the paper writes V = sgn(H); for ReLU this is read as the indicator of H > 0 (so that V (.) H is
+#     max(H, 0)); zeros of either sign and NaN give V = 0;
+#   * dropout: V = 1 (keep) with probability 1 - p, p = drop_threshold / 65536; element i is dropped iff its
+#     16-bit DIVRNG-v1 field (sample index 0, flat index i) is < drop_threshold.  As in the paper's algorithm
+#     there is no 1/(1-p) rescaling;
+#   * "(.)" with a 0/1 mask is a select: a masked position is +0.0 (inputs are finite);
+#   * packing: bit (i mod 32) of little-endian 32-bit word i // 32, unused high bits of the last word zero
+#     (the Q = 1 case of the packing rule above).
+def mask_bytes(total: int) -> int:
+    """Bytes of the packed mask of `total` elements: whole 32-bit words."""
+    return -(-int(total) // 32) * 4
+
+
+def pack_mask(v_flat: np.ndarray) -> np.ndarray:
+    return pack_codes(np.asarray(v_flat, dtype=np.uint8).reshape(-1), 1)
+
+
+def unpack_mask(words: np.ndarray, total: int) -> np.ndarray:
+    return unpack_codes(words, 1, total)
+
+
+def relu_forward(x: np.ndarray, x_dtype: str = F32):
+    """Forward of the "Relu operator": returns (H_out as fp32 values, packed mask words)."""
+    x32 = widen_input(x, x_dtype).reshape(-1)
+    v = (x32 > 0).astype(np.uint8)
+    out = np.where(v == 1, x32, np.float32(0)).astype(np.float32)
+    return out, pack_mask(v)
+
+
+def dropout_forward(x: np.ndarray, seed: int, drop_threshold: int, x_dtype: str = F32):
+    """Forward of the "Dropout operator" (no rescaling): returns (H_out as fp32 values, packed mask words)."""
+    if not 0 <= int(drop_threshold) <= 65536:
+        raise ValueError("drop_threshold must lie in [0, 65536]")
+    x32 = widen_input(x, x_dtype).reshape(-1)
+    fields = divrng_fields(seed, 0, np.arange(x32.size, dtype=np.uint64)).astype(np.uint32)
+    v = (fields >= np.uint32(drop_threshold)).astype(np.uint8)
+    out = np.where(v == 1, x32, np.float32(0)).astype(np.float32)
+    return out, pack_mask(v)
+
+
+def mask_backward(words: np.ndarray, grad_out: np.ndarray, x_dtype: str = F32) -> np.ndarray:
+    """Backward of both operators: grad_in = V (.) grad_out, as fp32 values."""
+    g32 = widen_input(grad_out, x_dtype).reshape(-1)
+    v = unpack_mask(words, g32.size)
+    return np.where(v == 1, g32, np.float32(0)).astype(np.float32)
