@@ -337,6 +337,46 @@ def run_ours(args):
                          "algorithmic_bytes_per_launch": pg_algo[pg_dom]},
         }
 
+    # ---- ReLU / dropout operators with a packed 1-bit mask, on the largest map of the set (this rank) ----
+    mask_ops = None
+    if not args.no_masks:
+        big = max(range(len(specs)), key=lambda i: dev_x[i].numel())
+        xs, ys = dev_x[big], dev_out[big]
+        total = xs.numel()
+        mbytes = binding.div_mask_bytes(total)
+        mbuf = torch.zeros(mbytes, dtype=torch.uint8, device=device)
+        # a second pair of buffers, so that successive calls do not find their input in the 126 MB L2
+        xs2, ys2 = torch.empty_like(xs).copy_(xs), torch.empty_like(xs)
+        pairs = [(xs, ys), (xs2, ys2)]
+        stream = binding.current_stream_handle()
+        dt = specs[big].x_dtype
+        calls = {
+            "relu_forward": lambda a, b: binding.div_relu_forward(a.data_ptr(), b.data_ptr(), mbuf.data_ptr(), mbytes, total, dt, stream),
+            "dropout_forward": lambda a, b: binding.div_dropout_forward(a.data_ptr(), b.data_ptr(), mbuf.data_ptr(), mbytes, total, 1, 6554, dt, stream),
+            "mask_backward": lambda a, b: binding.div_mask_backward(mbuf.data_ptr(), mbytes, a.data_ptr(), b.data_ptr(), total, dt, stream),
+        }
+        m_steps = max(4, min(args.steps, 50))
+        m_peak, m_peak_kind = measured_peak()
+        algo = 2 * total * xs.element_size() + total // 8
+        mask_ops = {"what": "mask operators on " + "x".join(map(str, specs[big].shape)) + " (two buffer pairs alternate: inputs never L2-resident)",
+                    "algorithmic_bytes_per_launch": algo, "steps": m_steps, "kernels": {}}
+        for name, fn in calls.items():
+            for k in range(3):
+                fn(*pairs[k % 2])
+            barrier()
+            evs = [(ev(), ev()) for _ in range(m_steps)]
+            for k in range(m_steps):
+                evs[k][0].record()
+                fn(*pairs[k % 2])
+                evs[k][1].record()
+            barrier()
+            us = statistics.mean(a.elapsed_time(b) for a, b in evs) * 1e3
+            gbs = algo / (us * 1e-6) / 1e9
+            mask_ops["kernels"][name] = {"us": round(us, 2), "roofline": {"bound": "hbm", "achieved": gbs, "peak": m_peak, "unit": "GB/s",
+                                                                         "frac": gbs / m_peak, "peak_kind": f"of {m_peak_kind}", "traffic": None}}
+        mask_ops["gpu_launches"] = 3 * (m_steps + 3)
+        del xs2, ys2
+
     ms_per_step = total_ms / args.steps
     job_ms, job_bytes = aggregate_over_ranks(ms_per_step, float(raw_bytes), dist if world > 1 else None, device)
     e2e_job_ms, _ = aggregate_over_ranks(e2e_ms, float(raw_bytes), dist if world > 1 else None, device)
@@ -386,6 +426,7 @@ def run_ours(args):
                                     "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": f"of {peak_kind}"},
         "cpu_baseline": cpu,
         "plane_groups": plane_groups,
+        "mask_ops": mask_ops,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
                 "steps": e2e_steps},
@@ -405,6 +446,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-plane-groups", action="store_true", help="skip the extra timed loop of the per-plane form")
+    ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
     ap.add_argument("--compress-flags", type=int, default=0,
                     help="DIV_FLAG_* bits passed to div_compress_ex (profiling aid: 4 = strip ring kernel instead of the lagged one)")

@@ -230,6 +230,30 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
    (total size a multiple of 4, planes up to 8192 elements), 0 general. */
 div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
 
+/*
+ * ReLU and dropout operators with a packed 1-bit mask (the paper's appendix algorithms "Relu operator" and
+ * "Dropout operator"; one bit per element, N^2/8 bytes per plane, in the byte count of Theorem 3A's proof):
+ *   forward   V = mask,  H_out = V (.) H_in,  V packed and cached          backward  grad_in = V (.) grad_out
+ * on flat arrays of `total` elements of `dtype` (1 <= total <= 2^40; DIV_ERR_SHAPE otherwise).
+ *   - ReLU: V = [H_in > 0] (the paper's sgn read as the indicator of positivity; zeros and NaN give 0);
+ *   - dropout: V = 1 (keep) with probability 1 - drop_threshold/65536: element i is dropped iff the 16-bit number of
+ *     the random stream described above for (seed, sample 0, flat index i) is < drop_threshold (0 <= drop_threshold
+ *     <= 65536, else DIV_ERR_PARAM); as in the paper's algorithm, kept values are not rescaled;
+ *   - "(.)" is a select: masked positions become +0.0;
+ *   - mask: bit (i mod 32) of little-endian 32-bit word i/32, ceil(total/32) words (div_mask_bytes), unused high
+ *     bits of the last word zero;
+ *   - x_dev / y_dev / grad_*_dev: device, `total` elements, 16-byte aligned; y_dev may be x_dev and grad_in_dev may
+ *     be grad_out_dev (in place); mask_dev: device, 16-byte aligned, at least div_mask_bytes bytes
+ *     (DIV_ERR_CAPACITY otherwise).  The calls enqueue one kernel on the stream and return.
+ */
+div_status div_mask_bytes(uint64_t total, uint64_t* out_bytes);
+div_status div_relu_forward(const void* x_dev, void* y_dev, void* mask_dev, size_t mask_capacity, uint64_t total,
+                            int32_t dtype, void* cuda_stream);
+div_status div_dropout_forward(const void* x_dev, void* y_dev, void* mask_dev, size_t mask_capacity, uint64_t total,
+                               int32_t dtype, uint64_t seed, uint32_t drop_threshold, void* cuda_stream);
+div_status div_mask_backward(const void* mask_dev, size_t mask_bytes, const void* grad_out_dev, void* grad_in_dev,
+                             uint64_t total, int32_t dtype, void* cuda_stream);
+
 /* Which kernels a descriptor maps to on the current device.  desc, out: host. */
 div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
 

@@ -24,6 +24,7 @@ DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 EXPORTED_SYMBOLS = (
     "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_debug_compress_starved",
     "div_decompress", "div_plan_query",
+    "div_mask_bytes", "div_relu_forward", "div_dropout_forward", "div_mask_backward",
     "div_planegroup_bytes", "div_planegroup_compress", "div_planegroup_decompress", "div_planegroup_plan_query",
     "div_read_device_status", "div_status_string",
 )
@@ -88,6 +89,15 @@ def lib() -> ctypes.CDLL:
         L.div_planegroup_decompress.restype = c_int32
         L.div_planegroup_plan_query.argtypes = L.div_plan_query.argtypes
         L.div_planegroup_plan_query.restype = c_int32
+        L.div_mask_bytes.argtypes = [c_uint64, ctypes.POINTER(c_uint64)]
+        L.div_mask_bytes.restype = c_int32
+        L.div_relu_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_size_t, c_uint64, c_int32, c_void_p]
+        L.div_relu_forward.restype = c_int32
+        L.div_dropout_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_size_t, c_uint64, c_int32, c_uint64, c_uint32,
+                                          c_void_p]
+        L.div_dropout_forward.restype = c_int32
+        L.div_mask_backward.argtypes = [c_void_p, c_size_t, c_void_p, c_void_p, c_uint64, c_int32, c_void_p]
+        L.div_mask_backward.restype = c_int32
         L.div_read_device_status.argtypes = [c_void_p, c_void_p, ctypes.POINTER(c_int32)]
         L.div_read_device_status.restype = c_int32
         L.div_status_string.argtypes = [c_int32]
@@ -176,6 +186,31 @@ def div_planegroup_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xha
     st = lib().div_planegroup_decompress(ctypes.byref(desc), c_void_p(comp_ptr), comp_bytes, c_void_p(xhat_ptr),
                                          c_void_p(stream))
     _check(st, "div_planegroup_decompress")
+
+
+def div_mask_bytes(total: int) -> int:
+    out = c_uint64(0)
+    _check(lib().div_mask_bytes(c_uint64(total), ctypes.byref(out)), "div_mask_bytes")
+    return out.value
+
+
+def div_relu_forward(x_ptr: int, y_ptr: int, mask_ptr: int, mask_capacity: int, total: int, dtype: str = "f32",
+                     stream: int = 0) -> None:
+    _check(lib().div_relu_forward(c_void_p(x_ptr), c_void_p(y_ptr), c_void_p(mask_ptr), mask_capacity, c_uint64(total),
+                                  DTYPE_CODES[dtype], c_void_p(stream)), "div_relu_forward")
+
+
+def div_dropout_forward(x_ptr: int, y_ptr: int, mask_ptr: int, mask_capacity: int, total: int, seed: int,
+                        drop_threshold: int, dtype: str = "f32", stream: int = 0) -> None:
+    _check(lib().div_dropout_forward(c_void_p(x_ptr), c_void_p(y_ptr), c_void_p(mask_ptr), mask_capacity, c_uint64(total),
+                                     DTYPE_CODES[dtype], c_uint64(seed & (2 ** 64 - 1)), c_uint32(drop_threshold),
+                                     c_void_p(stream)), "div_dropout_forward")
+
+
+def div_mask_backward(mask_ptr: int, mask_bytes: int, grad_out_ptr: int, grad_in_ptr: int, total: int,
+                      dtype: str = "f32", stream: int = 0) -> None:
+    _check(lib().div_mask_backward(c_void_p(mask_ptr), mask_bytes, c_void_p(grad_out_ptr), c_void_p(grad_in_ptr),
+                                   c_uint64(total), DTYPE_CODES[dtype], c_void_p(stream)), "div_mask_backward")
 
 
 def div_read_device_status(ws_ptr: int, stream: int = 0) -> int:

@@ -12,6 +12,7 @@
 #include "fused.cuh"
 #include "fused_v.cuh"
 #include "lagged.cuh"
+#include "masks.cuh"
 #include "planegroup.cuh"
 #include "planes.cuh"
 #include "twopass.cuh"
@@ -592,6 +593,74 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
             return launch_status();
         });
     });
+}
+
+// ------------------------------------------------------------------------------------------------
+// ReLU / dropout operators with a packed 1-bit mask
+// ------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+constexpr uint64_t MASK_MAX_TOTAL = 1ull << 40;
+inline uint64_t mask_bytes_of(uint64_t total) { return (total + 31) / 32 * 4; }
+
+div_status mask_forward(const void* x_dev, void* y_dev, void* mask_dev, size_t mask_capacity, uint64_t total,
+                        int32_t dtype, bool dropout, uint64_t seed, uint32_t drop_threshold, void* cuda_stream) {
+    if (!x_dev || !y_dev || !mask_dev) return DIV_ERR_NULL;
+    if (total < 1 || total > MASK_MAX_TOTAL) return DIV_ERR_SHAPE;
+    if (!(dtype == DIV_F32 || dtype == DIV_BF16) || drop_threshold > 65536u) return DIV_ERR_PARAM;
+    if (!aligned16(x_dev) || !aligned16(y_dev) || !aligned16(mask_dev)) return DIV_ERR_ALIGN;
+    if (mask_capacity < mask_bytes_of(total)) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    uint8_t* mask = (uint8_t*)mask_dev;
+    // the kernels store one byte per 8 elements: the rest of a partial last word is zero by contract
+    if (total % 32u != 0 && cudaMemsetAsync(mask + mask_bytes_of(total) - 4, 0, 4, stream) != cudaSuccess) return DIV_ERR_CUDA;
+    const unsigned grid = (unsigned)((total + 2047) / 2048);
+    const uint64_t base = rng_sample_base(seed, 0u);
+    if (dtype == DIV_F32) {
+        if (dropout) mask_forward_kernel<float, true><<<grid, 256, 0, stream>>>((const float*)x_dev, (float*)y_dev, mask, total, base, drop_threshold);
+        else mask_forward_kernel<float, false><<<grid, 256, 0, stream>>>((const float*)x_dev, (float*)y_dev, mask, total, base, 0u);
+    } else {
+        if (dropout) mask_forward_kernel<bf16, true><<<grid, 256, 0, stream>>>((const bf16*)x_dev, (bf16*)y_dev, mask, total, base, drop_threshold);
+        else mask_forward_kernel<bf16, false><<<grid, 256, 0, stream>>>((const bf16*)x_dev, (bf16*)y_dev, mask, total, base, 0u);
+    }
+    return launch_status();
+}
+}  // namespace
+
+extern "C" {
+
+div_status div_mask_bytes(uint64_t total, uint64_t* out_bytes) {
+    if (!out_bytes) return DIV_ERR_NULL;
+    if (total < 1 || total > MASK_MAX_TOTAL) return DIV_ERR_SHAPE;
+    *out_bytes = mask_bytes_of(total);
+    return DIV_OK;
+}
+
+div_status div_relu_forward(const void* x_dev, void* y_dev, void* mask_dev, size_t mask_capacity, uint64_t total,
+                            int32_t dtype, void* cuda_stream) {
+    return mask_forward(x_dev, y_dev, mask_dev, mask_capacity, total, dtype, false, 0, 0, cuda_stream);
+}
+
+div_status div_dropout_forward(const void* x_dev, void* y_dev, void* mask_dev, size_t mask_capacity, uint64_t total,
+                               int32_t dtype, uint64_t seed, uint32_t drop_threshold, void* cuda_stream) {
+    return mask_forward(x_dev, y_dev, mask_dev, mask_capacity, total, dtype, true, seed, drop_threshold, cuda_stream);
+}
+
+div_status div_mask_backward(const void* mask_dev, size_t mask_bytes, const void* grad_out_dev, void* grad_in_dev,
+                             uint64_t total, int32_t dtype, void* cuda_stream) {
+    if (!mask_dev || !grad_out_dev || !grad_in_dev) return DIV_ERR_NULL;
+    if (total < 1 || total > MASK_MAX_TOTAL) return DIV_ERR_SHAPE;
+    if (!(dtype == DIV_F32 || dtype == DIV_BF16)) return DIV_ERR_PARAM;
+    if (!aligned16(mask_dev) || !aligned16(grad_out_dev) || !aligned16(grad_in_dev)) return DIV_ERR_ALIGN;
+    if (mask_bytes < mask_bytes_of(total)) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const unsigned grid = (unsigned)((total + 2047) / 2048);
+    if (dtype == DIV_F32)
+        mask_backward_kernel<float><<<grid, 256, 0, stream>>>((const uint8_t*)mask_dev, (const float*)grad_out_dev, (float*)grad_in_dev, total);
+    else
+        mask_backward_kernel<bf16><<<grid, 256, 0, stream>>>((const uint8_t*)mask_dev, (const bf16*)grad_out_dev, (bf16*)grad_in_dev, total);
+    return launch_status();
 }
 
 div_status div_read_device_status(const void* workspace_dev, void* cuda_stream, int32_t* out_status) {

@@ -77,6 +77,23 @@ def test_planegroup_refuses_too_many_planes_and_bad_flags():
     assert L.div_planegroup_decompress(ctypes.byref(d), 16, 1 << 20, 34, None) == binding.DIV_ERR_ALIGN
 
 
+def test_mask_bytes_and_host_checks():
+    L = binding.lib()
+    for total in (1, 31, 32, 33, 49, 12544, 64 * 64 * 112 * 112):
+        assert binding.div_mask_bytes(total) == orc.mask_bytes(total)
+    out = ctypes.c_uint64(0)
+    assert L.div_mask_bytes(0, ctypes.byref(out)) == binding.DIV_ERR_SHAPE
+    assert L.div_mask_bytes((1 << 40) + 1, ctypes.byref(out)) == binding.DIV_ERR_SHAPE
+    assert L.div_mask_bytes(5, None) == binding.DIV_ERR_NULL
+    assert L.div_relu_forward(None, 16, 32, 64, 8, 0, None) == binding.DIV_ERR_NULL
+    assert L.div_relu_forward(16, 16, 32, 64, 8, 7, None) == binding.DIV_ERR_PARAM
+    assert L.div_relu_forward(16, 18, 32, 64, 8, 0, None) == binding.DIV_ERR_ALIGN
+    assert L.div_relu_forward(16, 16, 32, 3, 8, 0, None) == binding.DIV_ERR_CAPACITY
+    assert L.div_dropout_forward(16, 16, 32, 64, 8, 0, 1, 65537, None) == binding.DIV_ERR_PARAM
+    assert L.div_mask_backward(32, 3, 16, 16, 8, 0, None) == binding.DIV_ERR_CAPACITY
+    assert L.div_mask_backward(32, 64, 16, 16, 0, 0, None) == binding.DIV_ERR_SHAPE
+
+
 def test_bad_descriptors_are_refused_on_the_host():
     L = binding.lib()
     out = binding.DivLayout()
