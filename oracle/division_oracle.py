@@ -590,3 +590,63 @@ def mask_backward(words: np.ndarray, grad_out: np.ndarray, x_dtype: str = F32) -
     g32 = widen_input(grad_out, x_dtype).reshape(-1)
     v = unpack_mask(words, g32.size)
     return np.where(v == 1, g32, np.float32(0)).astype(np.float32)
+
+
+# ----------------------------------------------------------------------------------------
+# 1-D activation maps  (appendix "Compression of 1D and 3D Activation Maps": Minibatch x Channel x N,
+# average pooling and nearest up-sampling along the last axis, Quant and its inverse unchanged)
+# ----------------------------------------------------------------------------------------
+# Readings: as for 2-D maps.  A last block shorter than B is averaged over its in-bounds elements (the
+# paper's shapes use floor(N/B), which only covers N divisible by B); a block longer than the row is the
+# whole row; the block sum is the balanced pairwise tree over the B positions (neighbours first, positions
+# outside the row count as +0.0).  The random stream, packing and blob are those of the 2-D form with the
+# in-sample index e = c*N + i.
+def lfc_mean_1d(x32: np.ndarray, block: int) -> np.ndarray:
+    """H^L = AveragePooling1D(H), window = stride = B, for x32[M, C, N]; fp32 with the build's summation order."""
+    x32 = np.asarray(x32, dtype=np.float32)
+    m, c, n = x32.shape
+    block = min(int(block), n)
+    nb = -(-n // block)
+    xp = np.zeros((m, c, nb * block), dtype=np.float32)
+    xp[:, :, :n] = x32
+    total = _pairwise_tree_sum(xp.reshape(m, c, nb, block), axis=-1)
+    count = np.minimum(block, n - np.arange(nb) * block).astype(np.float32)
+    return (total / count[None, None]).astype(np.float32)
+
+
+def upsample_nearest_1d(lfc: np.ndarray, block: int, n: int) -> np.ndarray:
+    """UpSampling1D(H^L): position i takes the value of block i // B."""
+    return np.repeat(lfc, min(int(block), n), axis=2)[:, :, :n]
+
+
+def compress_1d(x: np.ndarray, block: int, qbits: int, seed: int,
+                x_dtype: str = F32, lfc_dtype: str = F32) -> Compressed:
+    """Forward-loop steps of Algorithm 1 for a 1-D activation map H of shape Minibatch x Channel x N."""
+    if qbits not in SUPPORTED_QBITS:
+        raise ValueError("Q must divide 32")
+    x32 = widen_input(x, x_dtype)
+    m, c, n = x32.shape
+    lfc = round_to_dtype(lfc_mean_1d(x32, block), lfc_dtype)
+    r = (x32 - upsample_nearest_1d(lfc, block, n)).reshape(m, c * n)
+    codes = np.empty((m, c * n), dtype=np.uint8)
+    delta = np.empty(m, dtype=np.float32)
+    step = np.empty(m, dtype=np.float32)
+    e = np.arange(c * n, dtype=np.uint64)
+    for i in range(m):
+        delta[i], step[i], scale = sample_stats(r[i], qbits)
+        codes[i] = quantize(r[i], delta[i], scale, divrng_fields(seed, i, e), qbits)
+    words = pack_codes(codes.reshape(-1), qbits)
+    layout = compressed_layout(m, c, 1, n, min(int(block), n), qbits, x_dtype, lfc_dtype)
+    return Compressed((m, c, 1, n), min(int(block), n), qbits, x_dtype, lfc_dtype, lfc[:, :, None, :], codes, words,
+                      delta, step, layout)
+
+
+def decompress_1d(comp: Compressed) -> np.ndarray:
+    """Backward-loop steps of Algorithm 1 for a 1-D map; returns fp32 values [M, C, N] rounded to the activation dtype."""
+    m, c, _, n = comp.shape
+    codes = unpack_codes(comp.words, comp.qbits, m * c * n).reshape(m, c * n)
+    hh = np.empty((m, c * n), dtype=np.float32)
+    for i in range(m):
+        hh[i] = dequantize(codes[i], comp.delta[i], comp.step[i])
+    xhat = upsample_nearest_1d(comp.lfc[:, :, 0, :], comp.block, n) + hh.reshape(m, c, n)
+    return round_to_dtype(xhat.astype(np.float32), comp.x_dtype)
