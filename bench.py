@@ -208,7 +208,7 @@ def run_ours(args):
     plans = [c.plan(args.compress_flags) for c in codecs]
     raw_bytes = sum(int(c.layout.raw_bytes) for c in codecs)
     comp_bytes = sum(int(c.layout.closed_form_bytes) for c in codecs)
-    kernels_per_step = sum((2 if p.fused in (0, 4) else 1) + 1 for p in plans)
+    kernels_per_step = sum((2 if p.fused in (0, 4, 5) else 1) + 1 for p in plans)
     torch.cuda.synchronize()
 
     def step(record=None):
@@ -389,7 +389,7 @@ def run_ours(args):
     algo_bytes = [int(c.layout.raw_bytes) + int(c.layout.closed_form_bytes) for c in codecs]
     comp_gbs = sum(algo_bytes) / (sum(comp_ms) * 1e-3) / 1e9
     dec_gbs = sum(algo_bytes) / (sum(dec_ms) * 1e-3) / 1e9
-    kernel_names = {4: "plane_stats_kernel + plane_quant_kernel", 3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
+    kernel_names = {5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel", 3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
     per_map = [{"map": "x".join(map(str, s.shape)), "compress_kernel": kernel_names[int(p.fused)],
                 "compress_us": round(cm * 1e3, 2), "compress_GBps": round(b / cm / 1e6, 1),
                 "decompress_us": round(dm * 1e3, 2), "decompress_GBps": round(b / dm / 1e6, 1)}

@@ -12,7 +12,9 @@
  *   decompress  H_hat = UpSampling(H^L) + Delta * V^H + delta                   (Sec. 4.2, Eq. 10)
  *
  * for an activation map H of shape N x C x H x W (the paper's Minibatch x Channel x N x N),
- * contiguous NCHW, fp32 or bf16.
+ * contiguous NCHW, fp32 or bf16.  A 1-D map (Minibatch x Channel x N; the appendix "Compression of 1D and 3D
+ * Activation Maps": pooling and up-sampling along the last axis) is described as N x C x 1 x W: a block then
+ * covers B consecutive elements of a row.  3-D maps are not supported.
  *
  * Conventions fixed by this library where the paper is silent (the same rules are written out in
  * the CPU checker, which was implemented separately):
@@ -95,7 +97,9 @@ typedef struct div_plan {
                                   choice from 40 MB up, and whenever the ring cannot hold a sample's share);
                                4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
                                   at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
-                               1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels */
+                               1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;
+                               5: 1-D maps (h == 1; the appendix on 1D and 3D activation maps), W%4==0, B a power of two
+                                  in [4,128], Q in {2,4,8}: two launches, the second read comes from L2 */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
     int32_t stages;         /* shared-memory ring depth (ring kernels only)                   */
@@ -114,6 +118,7 @@ typedef struct div_plan {
 #define DIV_FLAG_NO_STRIP_KERNEL 2u  /* never take the strip variant of the ring kernel    */
 #define DIV_FLAG_NO_LAGGED_KERNEL 4u /* never take the lagged (L2 re-read) kernel          */
 #define DIV_FLAG_NO_PLANE_KERNELS 8u /* never take the small-plane pair of kernels          */
+#define DIV_FLAG_NO_LINE_KERNELS 16u /* never take the pair of kernels for 1-D maps          */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:

@@ -12,6 +12,7 @@
 #include "fused.cuh"
 #include "fused_v.cuh"
 #include "lagged.cuh"
+#include "lines.cuh"
 #include "masks.cuh"
 #include "planegroup.cuh"
 #include "planes.cuh"
@@ -23,8 +24,8 @@ using namespace divk;
 typedef __nv_bfloat16 bf16;
 
 constexpr uint64_t SECTION_ALIGN = 128;
-constexpr uint32_t DIV_FLAG_ALL =
-    DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL | DIV_FLAG_NO_PLANE_KERNELS;
+constexpr uint32_t DIV_FLAG_ALL = DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL |
+                                  DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_NO_LINE_KERNELS;
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
@@ -206,16 +207,22 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     FusedPlan fp;
     VPlan vp;
     LPlan lp;
+    LineGeom lg;
+    const bool lines = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LINE_KERNELS)) && plan_lines(desc, s, &lg);
     const bool lag_first = prefer_lagged(desc, s);
-    const bool lag_ok = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
-    const bool vec_ok = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
+    const bool lag_ok = !lines && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
+    const bool vec_ok = !lines && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
     const bool lag = lag_ok && (lag_first || !vec_ok);
     const bool vec = vec_ok && !lag;
     PlaneGeom pg;
-    const bool planes = !lag && !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS)) && plan_planes(desc, s, &pg);
-    const bool fused = !lag && !vec && !planes && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
-    out->fused = lag ? 3 : (vec ? 2 : (planes ? 4 : (fused ? 1 : 0)));
-    if (lag) {
+    const bool planes = !lines && !lag && !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS)) && plan_planes(desc, s, &pg);
+    const bool fused = !lines && !lag && !vec && !planes && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
+    out->fused = lines ? 5 : (lag ? 3 : (vec ? 2 : (planes ? 4 : (fused ? 1 : 0))));
+    if (lines) {
+        out->grid = (int32_t)((lg.qps + 256 * LINE_QPT - 1) / (256 * LINE_QPT) * s.N);
+        out->threads = 256;
+        out->chunk_elems = 4 * LINE_QPT * 256;
+    } else if (lag) {
         out->grid = lp.grid;
         out->threads = lp.threads;
         out->stages = 0;
@@ -271,6 +278,10 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
         cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
         return DIV_ERR_CUDA;
+    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LINE_KERNELS))) {
+        LineGeom lg;
+        if (plan_lines(desc, s, &lg)) return compress_lines(desc, s, lo, lg, x_dev, blob, ws, seed, stream);
+    }
     const bool may_lag = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL));
     const bool may_strip = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL));
     LPlan lp;

@@ -1,0 +1,173 @@
+// Compress kernels for 1-D activation maps (the paper's appendix "Compression of 1D and 3D Activation Maps":
+// Minibatch x Channel x N, average pooling and nearest up-sampling along the last axis; Eq. 9 unchanged).
+// A 1-D map is described as N x C x 1 x W.  Conditions: W % 4 == 0, B a power of two in [4, 128], Q in {2, 4, 8}.
+//
+// Two launches, no dependency inside a kernel (token / MLP activations of one layer are tens of MB: the second
+// read of x comes from the 126 MB L2; larger tensors are still handled correctly, reading x twice from HBM):
+//   line_stats_kernel   a lane owns 4 consecutive elements; the B/4 lanes of a block meet through xor shuffles
+//                       (the balanced pairwise tree over the B positions, neighbours first); stored
+//                       low-frequency values; residual extremes -> per-sample min / max keys in the scratch slots
+//   line_quant_kernel   one thread per 4 consecutive elements (they share a block): Eq. 9 with stochastic
+//                       rounding on packed pairs, one byte / half-word / word of codes per thread and step
+#pragma once
+
+#include "fused_v.cuh"
+
+namespace divk {
+
+struct LineGeom {
+    uint32_t C, W, Wb, CHW;
+    uint32_t qpr;            // quads per row = W / 4
+    uint32_t cpr;            // warp chunks (32 quads) per row
+    uint32_t chunks;         // C * cpr: warp chunks per sample
+    uint32_t log2lpt;        // log2(B / 4): lanes per block
+    uint32_t B, tail_cnt;    // in-bounds elements of a row's last block
+    uint32_t qps;            // quads per sample
+    FastDiv by_cpr, by_qpr;
+};
+
+template <typename XT, typename LT>
+__global__ void __launch_bounds__(256)
+line_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, LineGeom g) {
+    const uint32_t n = blockIdx.y;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t lpt = 1u << g.log2lpt;
+    const XT* x_n = x + (size_t)n * g.CHW;
+    LT* lfc_n = lfc + (size_t)n * g.C * g.Wb;
+    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+    for (uint32_t wc = blockIdx.x * 8u + warp; wc < g.chunks; wc += gridDim.x * 8u) {
+        const uint32_t row = fdiv(wc, g.by_cpr);
+        const uint32_t q = (wc - row * g.cpr) * 32u + lane;          // quad inside the row
+        const bool ok = q < g.qpr;
+        uint64_t xy = 0ull, zw = 0ull;
+        if (ok) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + ((size_t)row * g.W + 4u * q)), xy, zw);
+        float a, b, c, d;
+        upk2(xy, a, b);
+        upk2(zw, c, d);
+        float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
+        for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+        const uint32_t t = q >> g.log2lpt;                            // block inside the row
+        const uint32_t cnt = (t + 1u == g.Wb) ? g.tail_cnt : g.B;
+        const float cntf = (float)cnt;
+        const float mean = ((cnt & (cnt - 1u)) == 0u) ? __fmul_rn(sum, __uint_as_float(0x7F000000u - __float_as_uint(cntf)))   // exact 1/2^k
+                                                      : __fdiv_rn(sum, cntf);
+        const float stored = Elem<LT>::round(mean);
+        if (ok) {
+            if ((q & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (size_t)row * g.Wb + t, mean);
+            // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
+            lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
+            hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
+        }
+    }
+    const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
+    const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+    if (lane == 0 && blockIdx.x * 8u + warp < g.chunks) {
+        uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+        atomicMax(slot + 0, kmin);
+        atomicMax(slot + 1, kmax);
+    }
+}
+
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+line_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const uint32_t* __restrict__ ws,
+                  void* __restrict__ packed_v, float* __restrict__ stats, LineGeom g, uint64_t seed) {
+    typedef typename PackedUnit<Q>::type OutT;
+    const uint32_t n = blockIdx.y;
+    const uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+    const QParams qp = make_qparams(key_float(~__ldg(slot + 0)), key_float(__ldg(slot + 1)), Q);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        stats[2 * (size_t)n + 0] = qp.delta;
+        stats[2 * (size_t)n + 1] = qp.step;
+    }
+    const uint64_t delta2 = pk2(qp.delta, qp.delta), scale2 = pk2(qp.scale, qp.scale);
+    const uint64_t base = rng_sample_base(seed, n);
+    const XT* x_n = x + (size_t)n * g.CHW;
+    const LT* lfc_n = lfc + (size_t)n * g.C * g.Wb;
+    OutT* packed = reinterpret_cast<OutT*>(packed_v) + (uint64_t)n * g.qps;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint64_t xy[QPT], zw[QPT];
+    float lf[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;                            // quad inside the sample
+        if (q < g.qps) {
+            StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy[k], zw[k]);
+            const uint32_t row = fdiv(q, g.by_qpr);
+            lf[k] = Elem<LT>::load(lfc_n + (size_t)row * g.Wb + ((q - row * g.qpr) >> g.log2lpt));
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < g.qps)
+            packed[q] = (OutT)quant_row<Q>(xy[k], zw[k], pk2(lf[k], lf[k]), delta2, scale2, rng_group(base, q));
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+constexpr int LINE_QPT = 4;
+
+inline bool plan_lines(const div_desc* d, const Shape& s, LineGeom* out) {
+    if (s.H != 1 || s.W % 4 != 0) return false;
+    if (!(d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return false;
+    if (s.B < 4 || s.B > 128 || (s.B & (s.B - 1)) != 0) return false;
+    if (s.CHW >= (1u << 31) || s.N > 65535u) return false;
+    LineGeom g;
+    g.C = s.C; g.W = s.W; g.Wb = s.Wb; g.CHW = s.CHW; g.B = s.B;
+    g.qpr = s.W / 4;
+    g.cpr = (g.qpr + 31u) / 32u;
+    const uint64_t chunks = (uint64_t)s.C * g.cpr;
+    if (chunks >= (1ull << 31)) return false;
+    g.chunks = (uint32_t)chunks;
+    g.log2lpt = 0;
+    while ((4u << g.log2lpt) < s.B) ++g.log2lpt;
+    g.tail_cnt = s.W - (s.Wb - 1u) * s.B;
+    g.qps = s.CHW / 4;
+    g.by_cpr = host_fastdiv(g.cpr);
+    g.by_qpr = host_fastdiv(g.qpr);
+    *out = g;
+    return true;
+}
+
+template <typename XT, typename LT>
+inline div_status compress_lines_t(const div_desc* d, const Shape& s, const div_layout& lo, const LineGeom& g,
+                                   const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+    const DeviceInfo di = device_info();
+    if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
+    // pass 1: enough CTAs per sample to fill the GPU a few times over, never more than there are warp chunks
+    uint32_t bx = (uint32_t)((16ull * di.sms + s.N - 1) / s.N);
+    const uint32_t bx_max = (g.chunks + 7u) / 8u;
+    if (bx > bx_max) bx = bx_max;
+    if (bx < 1) bx = 1;
+    const XT* xt = (const XT*)x;
+    LT* lfc = (LT*)(blob + lo.lfc_off);
+    line_stats_kernel<XT, LT><<<dim3(bx, s.N), 256, 0, st>>>(xt, lfc, ws, g);
+    if (cudaGetLastError() != cudaSuccess) return DIV_ERR_CUDA;
+    const uint32_t per_block = 256u * LINE_QPT;
+    const dim3 grid2((g.qps + per_block - 1) / per_block, s.N);
+    void* packed = blob + lo.packed_off;
+    float* stats = (float*)(blob + lo.stats_off);
+    switch (d->qbits) {
+        case 2: line_quant_kernel<XT, LT, 2, LINE_QPT><<<grid2, 256, 0, st>>>(xt, lfc, ws, packed, stats, g, seed); break;
+        case 4: line_quant_kernel<XT, LT, 4, LINE_QPT><<<grid2, 256, 0, st>>>(xt, lfc, ws, packed, stats, g, seed); break;
+        case 8: line_quant_kernel<XT, LT, 8, LINE_QPT><<<grid2, 256, 0, st>>>(xt, lfc, ws, packed, stats, g, seed); break;
+        default: return DIV_ERR_PARAM;
+    }
+    return cudaGetLastError() == cudaSuccess ? DIV_OK : DIV_ERR_CUDA;
+}
+
+inline div_status compress_lines(const div_desc* d, const Shape& s, const div_layout& lo, const LineGeom& g,
+                                 const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+    typedef __nv_bfloat16 bf16;
+    if (d->x_dtype == DIV_F32) {
+        if (d->lfc_dtype == DIV_F32) return compress_lines_t<float, float>(d, s, lo, g, x, blob, ws, seed, st);
+        return compress_lines_t<float, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+    }
+    if (d->lfc_dtype == DIV_F32) return compress_lines_t<bf16, float>(d, s, lo, g, x, blob, ws, seed, st);
+    return compress_lines_t<bf16, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+}
+
+}  // namespace divk
