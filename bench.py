@@ -198,6 +198,8 @@ def run_ours(args):
     build.build()
     binding.lib()
 
+    kernel_names_all = {5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel", 3: "lagged_kernel",
+                        2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
     specs = synth.config_specs(2)
     if args.maps:
         specs = [specs[int(i)] for i in args.maps.split(",")]
@@ -377,6 +379,59 @@ def run_ours(args):
         mask_ops["gpu_launches"] = 3 * (m_steps + 3)
         del xs2, ys2
 
+    # ---- 1-D maps (token activations; N x C x 1 x W descriptors), three transformer / MLP-shaped tensors ----
+    one_d = None
+    if not args.no_one_d:
+        shapes_1d = [("32x512x768 B=8 Q=4", (32, 512, 768), 8, 4), ("64x196x768 B=16 Q=2", (64, 196, 768), 16, 2),
+                     ("64x784x192 B=64 Q=2", (64, 784, 192), 64, 2)]
+        gen = torch.Generator(device=device).manual_seed(11)
+        t_x = [torch.randn(m, c, 1, n, device=device, generator=gen) for _, (m, c, n), _, _ in shapes_1d]
+        t_out = [torch.empty_like(x) for x in t_x]
+        t_codec = [binding.Codec(m, c, 1, n, b, q, device=device) for _, (m, c, n), b, q in shapes_1d]
+        t_steps = max(4, min(args.steps, 50))
+
+        def t_step(record=None):
+            for i, c in enumerate(t_codec):
+                if record is not None:
+                    record[0][i][0].record()
+                c.compress(t_x[i], seed=0)
+                if record is not None:
+                    record[0][i][1].record()
+            for i, c in enumerate(t_codec):
+                if record is not None:
+                    record[1][i][0].record()
+                c.decompress(out=t_out[i])
+                if record is not None:
+                    record[1][i][1].record()
+
+        for _ in range(3):
+            t_step()
+        barrier()
+        t_rec = [[[(ev(), ev()) for _ in t_codec] for _ in range(2)] for _ in range(t_steps)]
+        q0, q1 = ev(), ev()
+        q0.record()
+        for k in range(t_steps):
+            t_step(t_rec[k])
+        q1.record()
+        barrier()
+        t_ms = q0.elapsed_time(q1) / t_steps
+        t_raw = sum(int(c.layout.raw_bytes) for c in t_codec)
+        t_peak, t_peak_kind = measured_peak()
+        rows = []
+        for i, (name, _, _, _) in enumerate(shapes_1d):
+            cm = statistics.mean(t_rec[k][0][i][0].elapsed_time(t_rec[k][0][i][1]) for k in range(t_steps))
+            dm = statistics.mean(t_rec[k][1][i][0].elapsed_time(t_rec[k][1][i][1]) for k in range(t_steps))
+            b = int(t_codec[i].layout.raw_bytes) + int(t_codec[i].layout.closed_form_bytes)
+            rows.append({"map": name, "compress_kernel": kernel_names_all[int(t_codec[i].plan().fused)],
+                         "compress_us": round(cm * 1e3, 2), "compress_GBps": round(b / cm / 1e6, 1),
+                         "compress_frac_of_peak": round(b / cm / 1e6 / t_peak, 3),
+                         "decompress_us": round(dm * 1e3, 2), "decompress_GBps": round(b / dm / 1e6, 1),
+                         "decompress_frac_of_peak": round(b / dm / 1e6 / t_peak, 3)})
+        one_d = {"what": "1-D maps (Minibatch x Channel x N as N x C x 1 x W), compress then decompress of three tensors per step, this rank",
+                 "value": t_raw / (t_ms * 1e-3) / 1e9, "unit": UNIT, "steps": t_steps, "ms_per_step": t_ms,
+                 "peak": t_peak, "peak_kind": f"of {t_peak_kind}", "gpu_launches": 9 * (t_steps + 3), "per_map": rows}
+        del t_x, t_out, t_codec
+
     ms_per_step = total_ms / args.steps
     job_ms, job_bytes = aggregate_over_ranks(ms_per_step, float(raw_bytes), dist if world > 1 else None, device)
     e2e_job_ms, _ = aggregate_over_ranks(e2e_ms, float(raw_bytes), dist if world > 1 else None, device)
@@ -427,6 +482,7 @@ def run_ours(args):
         "cpu_baseline": cpu,
         "plane_groups": plane_groups,
         "mask_ops": mask_ops,
+        "one_d": one_d,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
                 "steps": e2e_steps},
@@ -446,6 +502,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-plane-groups", action="store_true", help="skip the extra timed loop of the per-plane form")
+    ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D maps")
     ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
     ap.add_argument("--compress-flags", type=int, default=0,

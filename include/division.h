@@ -108,8 +108,9 @@ typedef struct div_plan {
     int32_t smem_bytes;     /* dynamic shared memory per CTA                                  */
     int64_t chunk_elems;    /* elements per full chunk (ring kernels) or per unit (3)         */
     int64_t chunks_per_sample;
-    int32_t decompress_fast;/* 1: quad kernel (W%4==0, B a power of two >= 4); 2: flat kernel with a tile
-                               table (sample size a multiple of 4, planes up to 8192 elements); 0: general */
+    int32_t decompress_fast;/* 1: quad kernel (W%4==0, B a power of two >= 4); 3: the same conditions on a 1-D map
+                               (h == 1): line kernel; 2: flat kernel with a tile table (sample size a multiple of 4,
+                               planes up to 8192 elements); 0: general */
     int32_t reserved;
 } div_plan;
 

@@ -178,6 +178,51 @@ decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------
+// line kernel: 1-D maps (H == 1), W % 4 == 0, B a power of two >= 4.  One thread produces QPT quads, 256 quads
+// apart; a quad's block is (position in the row) / B.
+// grid = (ceil(quads_per_sample / (256*QPT)), N)
+// ---------------------------------------------------------------------------------------------
+struct DecLine {
+    uint32_t qps;        // quads per sample = C * W / 4
+    uint32_t C, Wb;
+    uint32_t qpr;        // quads per row
+    uint32_t log2lpt;    // log2(B / 4)
+    FastDiv by_qpr;
+};
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+decompress_line_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                       const float* __restrict__ stats, XT* __restrict__ xhat, DecLine d) {
+    __shared__ DeqTable<Q> table;
+    const uint32_t n = blockIdx.y;
+    table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
+    __syncthreads();
+    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
+    const LT* lfc_n = lfc + (size_t)n * d.C * d.Wb;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint32_t bits[QPT];
+    float lf[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < d.qps) {
+            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
+            const uint32_t row = fdiv(q, d.by_qpr);
+            lf[k] = Elem<LT>::load(lfc_n + (size_t)row * d.Wb + ((q - row * d.qpr) >> d.log2lpt));
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < d.qps) {
+            const float4 hq = table.quad(bits[k]);
+            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, __fadd_rn(lf[k], hq.x), __fadd_rn(lf[k], hq.y),
+                            __fadd_rn(lf[k], hq.z), __fadd_rn(lf[k], hq.w));
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // flat kernel: any W and B, sample size a multiple of 4 elements, planes of at most FLAT_MAX_HW
 // elements.  One thread produces QPT quads of 4 consecutive elements (global flat order), which may
 // lie in different tiles, rows or planes: the tile of every position of a plane comes from a table

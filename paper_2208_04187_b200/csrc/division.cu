@@ -254,7 +254,7 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
         out->grid = (int32_t)((s.tiles + 255) / 256);
         out->threads = 256;
     }
-    out->decompress_fast = decompress_fast_ok(s) ? 1 : (decompress_flat_ok(s) ? 2 : 0);
+    out->decompress_fast = decompress_fast_ok(s) ? ((s.H == 1 && s.CHW < (1u << 31)) ? 3 : 1) : (decompress_flat_ok(s) ? 2 : 0);
     return DIV_OK;
 }
 
@@ -357,7 +357,19 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
             const LT* lfc = (const LT*)(blob + lo.lfc_off);
             const uint32_t* packed = (const uint32_t*)(blob + lo.packed_off);
             const float* stats = (const float*)(blob + lo.stats_off);
-            if (decompress_fast_ok(s)) {
+            if (decompress_fast_ok(s) && s.H == 1 && s.CHW < (1u << 31)) {
+                DecLine d;
+                d.qps = s.CHW / 4;
+                d.C = s.C;
+                d.Wb = s.Wb;
+                d.qpr = s.W / 4;
+                d.log2lpt = 0;
+                while ((4u << d.log2lpt) < s.B) ++d.log2lpt;
+                d.by_qpr = make_fastdiv(d.qpr);
+                const uint32_t per_block = 256u * DEC_QPT;
+                dim3 grid((d.qps + per_block - 1) / per_block, s.N);
+                decompress_line_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+            } else if (decompress_fast_ok(s)) {
                 DecFast d;
                 d.qps = s.CHW / 4;
                 d.C = s.C;

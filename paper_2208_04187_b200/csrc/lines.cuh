@@ -26,6 +26,8 @@ struct LineGeom {
     FastDiv by_cpr, by_qpr;
 };
 
+constexpr int LINE_U = 4;     // warp chunks a warp works on at a time (their loads are issued together)
+
 template <typename XT, typename LT>
 __global__ void __launch_bounds__(256)
 line_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, LineGeom g) {
@@ -35,35 +37,47 @@ line_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
     const XT* x_n = x + (size_t)n * g.CHW;
     LT* lfc_n = lfc + (size_t)n * g.C * g.Wb;
     float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-    for (uint32_t wc = blockIdx.x * 8u + warp; wc < g.chunks; wc += gridDim.x * 8u) {
-        const uint32_t row = fdiv(wc, g.by_cpr);
-        const uint32_t q = (wc - row * g.cpr) * 32u + lane;          // quad inside the row
-        const bool ok = q < g.qpr;
-        uint64_t xy = 0ull, zw = 0ull;
-        if (ok) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + ((size_t)row * g.W + 4u * q)), xy, zw);
-        float a, b, c, d;
-        upk2(xy, a, b);
-        upk2(zw, c, d);
-        float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
-        for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-        const uint32_t t = q >> g.log2lpt;                            // block inside the row
-        const uint32_t cnt = (t + 1u == g.Wb) ? g.tail_cnt : g.B;
-        const float cntf = (float)cnt;
-        const float mean = ((cnt & (cnt - 1u)) == 0u) ? __fmul_rn(sum, __uint_as_float(0x7F000000u - __float_as_uint(cntf)))   // exact 1/2^k
-                                                      : __fdiv_rn(sum, cntf);
-        const float stored = Elem<LT>::round(mean);
-        if (ok) {
-            if ((q & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (size_t)row * g.Wb + t, mean);
-            // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
-            lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
-            hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
+    for (uint32_t wg = blockIdx.x * 8u + warp; wg * LINE_U < g.chunks; wg += gridDim.x * 8u) {
+        uint64_t xy[LINE_U], zw[LINE_U];
+        uint32_t row[LINE_U], q[LINE_U];
+        bool ok[LINE_U];
+#pragma unroll
+        for (int u = 0; u < LINE_U; ++u) {
+            const uint32_t wc = wg * LINE_U + u;
+            const bool live = wc < g.chunks;
+            row[u] = fdiv(live ? wc : 0u, g.by_cpr);
+            q[u] = ((live ? wc : 0u) - row[u] * g.cpr) * 32u + lane;          // quad inside the row
+            ok[u] = live && q[u] < g.qpr;
+            xy[u] = 0ull;
+            zw[u] = 0ull;
+            if (ok[u]) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + ((size_t)row[u] * g.W + 4u * q[u])), xy[u], zw[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < LINE_U; ++u) {
+            float a, b, c, d;
+            upk2(xy[u], a, b);
+            upk2(zw[u], c, d);
+            float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
+            for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+            const uint32_t t = q[u] >> g.log2lpt;                         // block inside the row
+            const uint32_t cnt = (t + 1u == g.Wb) ? g.tail_cnt : g.B;
+            const float cntf = (float)cnt;
+            const float mean = ((cnt & (cnt - 1u)) == 0u) ? __fmul_rn(sum, __uint_as_float(0x7F000000u - __float_as_uint(cntf)))   // exact 1/2^k
+                                                          : __fdiv_rn(sum, cntf);
+            const float stored = Elem<LT>::round(mean);
+            if (ok[u]) {
+                if ((q[u] & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (size_t)row[u] * g.Wb + t, mean);
+                // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
+                lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
+                hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
+            }
         }
     }
     const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
     const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
-    if (lane == 0 && blockIdx.x * 8u + warp < g.chunks) {
+    if (lane == 0) {
         uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
-        atomicMax(slot + 0, kmin);
+        atomicMax(slot + 0, kmin);       // neutral keys when this warp had no chunk
         atomicMax(slot + 1, kmax);
     }
 }
@@ -139,7 +153,7 @@ inline div_status compress_lines_t(const div_desc* d, const Shape& s, const div_
     if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
     // pass 1: enough CTAs per sample to fill the GPU a few times over, never more than there are warp chunks
     uint32_t bx = (uint32_t)((16ull * di.sms + s.N - 1) / s.N);
-    const uint32_t bx_max = (g.chunks + 7u) / 8u;
+    const uint32_t bx_max = (g.chunks + 8u * LINE_U - 1u) / (8u * LINE_U);
     if (bx > bx_max) bx = bx_max;
     if (bx < 1) bx = 1;
     const XT* xt = (const XT*)x;
