@@ -208,7 +208,7 @@ decompress_line_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
         if (q < d.qps) {
             bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
             const uint32_t row = fdiv(q, d.by_qpr);
-            lf[k] = Elem<LT>::load(lfc_n + (size_t)row * d.Wb + ((q - row * d.qpr) >> d.log2lpt));
+            lf[k] = Elem<LT>::load(lfc_n + (row * d.Wb + ((q - row * d.qpr) >> d.log2lpt)));
         }
     }
 #pragma unroll

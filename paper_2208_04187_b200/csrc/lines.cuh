@@ -22,6 +22,8 @@ struct LineGeom {
     uint32_t chunks;         // C * cpr: warp chunks per sample
     uint32_t log2lpt;        // log2(B / 4): lanes per block
     uint32_t B, tail_cnt;    // in-bounds elements of a row's last block
+    float inv_full, inv_tail;   // 1 / count of a full block and of a row's last block when that is a power of two, else 0
+    float cnt_full, cnt_tail;
     uint32_t qps;            // quads per sample
     FastDiv by_cpr, by_qpr;
 };
@@ -50,7 +52,7 @@ line_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
             ok[u] = live && q[u] < g.qpr;
             xy[u] = 0ull;
             zw[u] = 0ull;
-            if (ok[u]) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + ((size_t)row[u] * g.W + 4u * q[u])), xy[u], zw[u]);
+            if (ok[u]) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (row[u] * g.W + 4u * q[u])), xy[u], zw[u]);   // < CHW < 2^31
         }
 #pragma unroll
         for (int u = 0; u < LINE_U; ++u) {
@@ -60,13 +62,12 @@ line_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
             float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
             for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
             const uint32_t t = q[u] >> g.log2lpt;                         // block inside the row
-            const uint32_t cnt = (t + 1u == g.Wb) ? g.tail_cnt : g.B;
-            const float cntf = (float)cnt;
-            const float mean = ((cnt & (cnt - 1u)) == 0u) ? __fmul_rn(sum, __uint_as_float(0x7F000000u - __float_as_uint(cntf)))   // exact 1/2^k
-                                                          : __fdiv_rn(sum, cntf);
+            const bool tail = t + 1u == g.Wb;
+            const float inv = tail ? g.inv_tail : g.inv_full;
+            const float mean = (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, tail ? g.cnt_tail : g.cnt_full);
             const float stored = Elem<LT>::round(mean);
             if (ok[u]) {
-                if ((q[u] & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (size_t)row[u] * g.Wb + t, mean);
+                if ((q[u] & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (row[u] * g.Wb + t), mean);
                 // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
                 lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
                 hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
@@ -106,9 +107,9 @@ line_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const ui
     for (int k = 0; k < QPT; ++k) {
         const uint32_t q = q0 + k * 256u;                            // quad inside the sample
         if (q < g.qps) {
-            StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy[k], zw[k]);
+            StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + q * 4u), xy[k], zw[k]);
             const uint32_t row = fdiv(q, g.by_qpr);
-            lf[k] = Elem<LT>::load(lfc_n + (size_t)row * g.Wb + ((q - row * g.qpr) >> g.log2lpt));
+            lf[k] = Elem<LT>::load(lfc_n + (row * g.Wb + ((q - row * g.qpr) >> g.log2lpt)));
         }
     }
 #pragma unroll
@@ -139,6 +140,10 @@ inline bool plan_lines(const div_desc* d, const Shape& s, LineGeom* out) {
     g.log2lpt = 0;
     while ((4u << g.log2lpt) < s.B) ++g.log2lpt;
     g.tail_cnt = s.W - (s.Wb - 1u) * s.B;
+    g.cnt_full = (float)s.B;
+    g.cnt_tail = (float)g.tail_cnt;
+    g.inv_full = 1.0f / (float)s.B;                                                   // B is a power of two: exact
+    g.inv_tail = (g.tail_cnt & (g.tail_cnt - 1u)) == 0u ? 1.0f / (float)g.tail_cnt : 0.f;
     g.qps = s.CHW / 4;
     g.by_cpr = host_fastdiv(g.cpr);
     g.by_qpr = host_fastdiv(g.qpr);
