@@ -176,6 +176,67 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def measure_train_step(device, ev, barrier, batch=64, steps=3):
+    """Forward + backward of a randomly initialised torchvision ResNet-50 on synthetic images, with plain autograd
+    and with the activation cache of Algorithm 1; memory in the paper's way (allocated after forward minus after
+    backward), time with CUDA events.  The model is a stand-in for the paper's workload; its kernels are torch's."""
+    import torch
+    import torchvision
+
+    from paper_2208_04187_b200 import autograd as dv
+
+    torch.manual_seed(0)
+    x = torch.randn(batch, 3, 224, 224, device=device)
+
+    def run(model, make_cache):
+        model.zero_grad(set_to_none=True)
+        barrier()
+        base = torch.cuda.memory_allocated(device)
+        t0, t1 = ev(), ev()
+        t0.record()
+        cache = make_cache()
+        if cache is None:
+            loss = model(x).square().mean()
+        else:
+            with cache:
+                loss = model(x).square().mean()
+        barrier()
+        after_fwd = torch.cuda.memory_allocated(device)
+        loss.backward()
+        t1.record()
+        barrier()
+        after_bwd = torch.cuda.memory_allocated(device)
+        grads = sum(p.grad.numel() * p.grad.element_size() for p in model.parameters() if p.grad is not None)
+        del loss
+        return {"ms": t0.elapsed_time(t1), "activation_bytes": after_fwd - base, "after_bwd_minus_grads": after_bwd - base - grads,
+                "cache": cache}
+
+    out = {}
+    for name in ("plain", "division"):
+        model = torchvision.models.resnet50(weights=None).to(device).train()
+        make_cache = lambda: None
+        if name == "division":
+            dv.to_division_modules(model)
+            make_cache = lambda: dv.DivisionCache(block=8, qbits=2, seed=1)
+        for _ in range(2):
+            run(model, make_cache)
+        rs = [run(model, make_cache) for _ in range(steps)]
+        out[name] = {"ms_per_step": statistics.mean(r["ms"] for r in rs),
+                     "activation_bytes_after_forward": int(statistics.mean(r["activation_bytes"] for r in rs))}
+        if name == "division":
+            c = rs[-1]["cache"]
+            out[name].update({"maps_compressed": c.maps, "raw_bytes_of_those_maps": c.raw_bytes, "cached_bytes": c.cached_bytes,
+                              "ratio_of_those_maps": c.raw_bytes / max(c.cached_bytes, 1)})
+        del model, rs
+        torch.cuda.empty_cache()
+    out["what"] = (f"torchvision ResNet-50 (random init), batch {batch} x 3 x 224 x 224 fp32 synthetic, forward + backward; "
+                   "activation bytes = allocated after forward - before the step (the paper's MEM_after_fwd - MEM_after_bwd, "
+                   "gradients excluded); division = DivisionCache(B=8, Q=2) + ReLU with packed 1-bit masks")
+    out["activation_memory_ratio"] = out["plain"]["activation_bytes_after_forward"] / max(out["division"]["activation_bytes_after_forward"], 1)
+    out["time_ratio_division_over_plain"] = out["division"]["ms_per_step"] / out["plain"]["ms_per_step"]
+    return out
+
+
 # ----------------------------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------------------------
@@ -432,6 +493,20 @@ def run_ours(args):
                  "peak": t_peak, "peak_kind": f"of {t_peak_kind}", "gpu_launches": 9 * (t_steps + 3), "per_map": rows}
         del t_x, t_out, t_codec
 
+    # ---- Algorithm 1 around a synthetic ResNet-50 step: activation memory (after forward - after backward) and
+    # ---- forward+backward time, plain autograd against the cache (B=8, Q=2; ReLU with packed masks) ----
+    train_step = None
+    if not args.no_train_step and not args.maps:
+        dev_x.clear()                   # hand the benchmark's device buffers back before the model allocates
+        dev_out.clear()
+        for c in codecs:
+            c.blob = c.workspace = None
+        torch.cuda.empty_cache()
+        try:
+            train_step = measure_train_step(device, ev, barrier)
+        except Exception as exc:       # the headline line must not depend on torchvision or on free memory
+            train_step = {"error": f"{type(exc).__name__}: {exc}"}
+
     ms_per_step = total_ms / args.steps
     job_ms, job_bytes = aggregate_over_ranks(ms_per_step, float(raw_bytes), dist if world > 1 else None, device)
     e2e_job_ms, _ = aggregate_over_ranks(e2e_ms, float(raw_bytes), dist if world > 1 else None, device)
@@ -483,6 +558,7 @@ def run_ours(args):
         "plane_groups": plane_groups,
         "mask_ops": mask_ops,
         "one_d": one_d,
+        "train_step": train_step,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
                 "steps": e2e_steps},
@@ -502,6 +578,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-plane-groups", action="store_true", help="skip the extra timed loop of the per-plane form")
+    ap.add_argument("--no-train-step", action="store_true", help="skip the ResNet-50 forward+backward memory / time measurement")
     ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D maps")
     ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
