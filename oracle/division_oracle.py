@@ -650,3 +650,111 @@ def decompress_1d(comp: Compressed) -> np.ndarray:
         hh[i] = dequantize(codes[i], comp.delta[i], comp.step[i])
     xhat = upsample_nearest_1d(comp.lfc[:, :, 0, :], comp.block, n) + hh.reshape(m, c, n)
     return round_to_dtype(xhat.astype(np.float32), comp.x_dtype)
+
+
+# ----------------------------------------------------------------------------------------
+# 3-D activation maps  (appendix "Compression of 1D and 3D Activation Maps": Minibatch x Channel x N x N x N,
+# average pooling and nearest up-sampling over B x B x B blocks, Quant and its inverse unchanged)
+# ----------------------------------------------------------------------------------------
+# Readings as for 2-D maps: ceil grid on every axis, a partial block is averaged over its in-bounds elements, a
+# block larger than all three sides behaves like a block equal to the largest side; the block sum is the balanced
+# pairwise tree along the depth axis first, then down the rows, then across the columns (positions outside the map
+# count as +0.0; for depth 1 this is the 2-D order).  In-sample index e = ((c*D + d)*H + h)*W + w; random stream,
+# packing and blob as before, with N*C*ceil(D/B)*ceil(H/B)*ceil(W/B) low-frequency values.
+def _block3(d: int, h: int, w: int, block: int) -> int:
+    return min(int(block), max(d, h, w))
+
+
+def lfc_mean_3d(x32: np.ndarray, block: int) -> np.ndarray:
+    """H^L = AveragePooling3D(H), window = stride = B, for x32[M, C, D, H, W]; fp32, the build's summation order."""
+    x32 = np.asarray(x32, dtype=np.float32)
+    m, c, d, h, w = x32.shape
+    b = _block3(d, h, w, block)
+    db, hb, wb = -(-d // b), -(-h // b), -(-w // b)
+    xp = np.zeros((m, c, db * b, hb * b, wb * b), dtype=np.float32)
+    xp[:, :, :d, :h, :w] = x32
+    t = xp.reshape(m, c, db, b, hb, b, wb, b).transpose(0, 1, 2, 4, 6, 3, 5, 7)      # [..., depth, row, col] per block
+    s = _pairwise_tree_sum(t, axis=-3)          # along the depth of every (row, col) position
+    s = _pairwise_tree_sum(s, axis=-2)          # down the rows
+    s = _pairwise_tree_sum(s, axis=-1)          # across the columns
+    nd = np.minimum(b, d - np.arange(db) * b)
+    nh = np.minimum(b, h - np.arange(hb) * b)
+    nw = np.minimum(b, w - np.arange(wb) * b)
+    count = (nd[:, None, None] * nh[None, :, None] * nw[None, None, :]).astype(np.float32)
+    return (s / count[None, None]).astype(np.float32)
+
+
+def upsample_nearest_3d(lfc: np.ndarray, block: int, d: int, h: int, w: int) -> np.ndarray:
+    b = _block3(d, h, w, block)
+    up = np.repeat(np.repeat(np.repeat(lfc, b, axis=2), b, axis=3), b, axis=4)
+    return up[:, :, :d, :h, :w]
+
+
+@dataclass
+class Compressed3D:
+    shape: tuple           # (M, C, D, H, W)
+    block: int
+    qbits: int
+    x_dtype: str
+    lfc_dtype: str
+    lfc: np.ndarray        # [M, C, Db, Hb, Wb] fp32 values as stored
+    codes: np.ndarray      # [M, C*D*H*W]
+    words: np.ndarray
+    delta: np.ndarray
+    step: np.ndarray
+    layout: Layout
+
+    def blob(self) -> np.ndarray:
+        out = np.zeros(self.layout.total_bytes, dtype=np.uint8)
+        raw = self.lfc.astype("<f4").tobytes() if self.lfc_dtype == F32 else f32_to_bf16_bits(self.lfc).astype("<u2").tobytes()
+        lo = self.layout
+        out[lo.lfc_off:lo.lfc_off + lo.lfc_bytes] = np.frombuffer(raw, dtype=np.uint8)
+        out[lo.packed_off:lo.packed_off + lo.packed_bytes] = np.frombuffer(self.words.astype("<u4").tobytes(), dtype=np.uint8)
+        stats = np.stack([self.delta, self.step], axis=1).astype("<f4")
+        out[lo.stats_off:lo.stats_off + lo.stats_bytes] = np.frombuffer(stats.tobytes(), dtype=np.uint8)
+        return out
+
+
+def layout_3d(m: int, c: int, d: int, h: int, w: int, block: int, qbits: int,
+              x_dtype: str = F32, lfc_dtype: str = F32) -> Layout:
+    b = _block3(d, h, w, block)
+    tiles = m * c * (-(-d // b)) * (-(-h // b)) * (-(-w // b))
+    lfc_bytes = tiles * _DTYPE_BYTES[lfc_dtype]
+    packed_bytes = -(-(m * c * d * h * w * qbits) // 32) * 4
+    packed_off = _align(lfc_bytes, SECTION_ALIGN)
+    stats_off = _align(packed_off + packed_bytes, SECTION_ALIGN)
+    return Layout(0, lfc_bytes, packed_off, packed_bytes, stats_off, 8 * m, stats_off + 8 * m,
+                  lfc_bytes + packed_bytes + 8 * m, m * c * d * h * w * _DTYPE_BYTES[x_dtype])
+
+
+def compress_3d(x: np.ndarray, block: int, qbits: int, seed: int,
+                x_dtype: str = F32, lfc_dtype: str = F32) -> Compressed3D:
+    """Forward-loop steps of Algorithm 1 for a 3-D activation map H of shape Minibatch x Channel x D x H x W."""
+    if qbits not in SUPPORTED_QBITS:
+        raise ValueError("Q must divide 32")
+    x32 = widen_input(x, x_dtype)
+    m, c, d, h, w = x32.shape
+    per = c * d * h * w
+    lfc = round_to_dtype(lfc_mean_3d(x32, block), lfc_dtype)
+    r = (x32 - upsample_nearest_3d(lfc, block, d, h, w)).reshape(m, per)
+    codes = np.empty((m, per), dtype=np.uint8)
+    delta = np.empty(m, dtype=np.float32)
+    step = np.empty(m, dtype=np.float32)
+    e = np.arange(per, dtype=np.uint64)
+    for i in range(m):
+        delta[i], step[i], scale = sample_stats(r[i], qbits)
+        codes[i] = quantize(r[i], delta[i], scale, divrng_fields(seed, i, e), qbits)
+    words = pack_codes(codes.reshape(-1), qbits)
+    return Compressed3D((m, c, d, h, w), _block3(d, h, w, block), qbits, x_dtype, lfc_dtype, lfc, codes, words, delta, step,
+                        layout_3d(m, c, d, h, w, block, qbits, x_dtype, lfc_dtype))
+
+
+def decompress_3d(comp: Compressed3D) -> np.ndarray:
+    m, c, d, h, w = comp.shape
+    per = c * d * h * w
+    codes = unpack_codes(comp.words, comp.qbits, m * per).reshape(m, per)
+    hh = np.empty((m, per), dtype=np.float32)
+    for i in range(m):
+        hh[i] = dequantize(codes[i], comp.delta[i], comp.step[i])
+    xhat = upsample_nearest_3d(comp.lfc, comp.block, d, h, w) + hh.reshape(m, c, d, h, w)
+    return round_to_dtype(xhat.astype(np.float32), comp.x_dtype)
