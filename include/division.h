@@ -14,7 +14,7 @@
  * for an activation map H of shape N x C x H x W (the paper's Minibatch x Channel x N x N),
  * contiguous NCHW, fp32 or bf16.  A 1-D map (Minibatch x Channel x N; the appendix "Compression of 1D and 3D
  * Activation Maps": pooling and up-sampling along the last axis) is described as N x C x 1 x W: a block then
- * covers B consecutive elements of a row.  3-D maps are not supported.
+ * covers B consecutive elements of a row.  3-D maps have entry points of their own (div_compress_3d).
  *
  * Conventions fixed by this library where the paper is silent (the same rules are written out in
  * the CPU checker, which was implemented separately):
@@ -235,6 +235,27 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
    {2,4,8}, sample size a multiple of 4), 0 general kernel; plan.decompress_fast: 1 quad kernel, 2 flat kernel
    (total size a multiple of 4, planes up to 8192 elements), 0 general. */
 div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_plan* out);
+
+/*
+ * 3-D activation maps (the appendix "Compression of 1D and 3D Activation Maps": Minibatch x Channel x N x N x N;
+ * average pooling and nearest up-sampling over B x B x B blocks, Eq. 9 and its inverse unchanged).  x is
+ * contiguous N x C x D x H x W.  Conventions as for 2-D maps: ceil grid on every axis, partial blocks average their
+ * in-bounds elements, a block larger than every side is the largest side; the block sum is the balanced pairwise
+ * tree along the depth axis, then down the rows, then across the columns; in-sample index
+ * e = ((c*D + d)*H + h)*W + w; one fp32 (delta, Delta) pair per sample; blob = [lfc: N*C*ceil(D/B)*ceil(H/B)*
+ * ceil(W/B) values | packed | stats] with the same padding, workspace as for div_compress.  c*d*h*w < 2^32.
+ * General kernels only (one thread per block, then one per packed word): any shape, block size and Q.
+ * Arguments, ownership and error codes as for div_compressed_bytes / div_compress / div_decompress.
+ */
+typedef struct div_desc3d {
+    int64_t n, c, d, h, w;
+    int32_t block, qbits, x_dtype, lfc_dtype;
+} div_desc3d;
+div_status div_compressed_bytes_3d(const div_desc3d* desc, div_layout* out);
+div_status div_compress_3d(const div_desc3d* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                           void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream);
+div_status div_decompress_3d(const div_desc3d* desc, const void* comp_dev, size_t comp_bytes, void* xhat_dev,
+                             void* cuda_stream);
 
 /*
  * ReLU and dropout operators with a packed 1-bit mask (the paper's appendix algorithms "Relu operator" and

@@ -25,6 +25,7 @@ DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 EXPORTED_SYMBOLS = (
     "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_debug_compress_starved",
     "div_decompress", "div_plan_query",
+    "div_compressed_bytes_3d", "div_compress_3d", "div_decompress_3d",
     "div_mask_bytes", "div_relu_forward", "div_dropout_forward", "div_mask_backward",
     "div_planegroup_bytes", "div_planegroup_compress", "div_planegroup_decompress", "div_planegroup_plan_query",
     "div_read_device_status", "div_status_string",
@@ -33,6 +34,11 @@ EXPORTED_SYMBOLS = (
 
 class DivDesc(ctypes.Structure):
     _fields_ = [("n", c_int64), ("c", c_int64), ("h", c_int64), ("w", c_int64),
+                ("block", c_int32), ("qbits", c_int32), ("x_dtype", c_int32), ("lfc_dtype", c_int32)]
+
+
+class DivDesc3D(ctypes.Structure):
+    _fields_ = [("n", c_int64), ("c", c_int64), ("d", c_int64), ("h", c_int64), ("w", c_int64),
                 ("block", c_int32), ("qbits", c_int32), ("x_dtype", c_int32), ("lfc_dtype", c_int32)]
 
 
@@ -90,6 +96,13 @@ def lib() -> ctypes.CDLL:
         L.div_planegroup_decompress.restype = c_int32
         L.div_planegroup_plan_query.argtypes = L.div_plan_query.argtypes
         L.div_planegroup_plan_query.restype = c_int32
+        L.div_compressed_bytes_3d.argtypes = [ctypes.POINTER(DivDesc3D), ctypes.POINTER(DivLayout)]
+        L.div_compressed_bytes_3d.restype = c_int32
+        L.div_compress_3d.argtypes = [ctypes.POINTER(DivDesc3D), c_void_p, c_void_p, c_size_t, c_void_p, c_size_t, c_uint64,
+                                      c_void_p]
+        L.div_compress_3d.restype = c_int32
+        L.div_decompress_3d.argtypes = [ctypes.POINTER(DivDesc3D), c_void_p, c_size_t, c_void_p, c_void_p]
+        L.div_decompress_3d.restype = c_int32
         L.div_mask_bytes.argtypes = [c_uint64, ctypes.POINTER(c_uint64)]
         L.div_mask_bytes.restype = c_int32
         L.div_relu_forward.argtypes = [c_void_p, c_void_p, c_void_p, c_size_t, c_uint64, c_int32, c_void_p]
@@ -187,6 +200,27 @@ def div_planegroup_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xha
     st = lib().div_planegroup_decompress(ctypes.byref(desc), c_void_p(comp_ptr), comp_bytes, c_void_p(xhat_ptr),
                                          c_void_p(stream))
     _check(st, "div_planegroup_decompress")
+
+
+def make_desc_3d(n, c, d, h, w, block, qbits, x_dtype="f32", lfc_dtype="f32") -> DivDesc3D:
+    return DivDesc3D(int(n), int(c), int(d), int(h), int(w), int(block), int(qbits), DTYPE_CODES[x_dtype], DTYPE_CODES[lfc_dtype])
+
+
+def div_compressed_bytes_3d(desc: DivDesc3D) -> DivLayout:
+    out = DivLayout()
+    _check(lib().div_compressed_bytes_3d(ctypes.byref(desc), ctypes.byref(out)), "div_compressed_bytes_3d")
+    return out
+
+
+def div_compress_3d(desc: DivDesc3D, x_ptr: int, comp_ptr: int, comp_capacity: int, ws_ptr: int, ws_bytes: int,
+                    seed: int, stream: int = 0) -> None:
+    _check(lib().div_compress_3d(ctypes.byref(desc), c_void_p(x_ptr), c_void_p(comp_ptr), comp_capacity, c_void_p(ws_ptr),
+                                 ws_bytes, c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream)), "div_compress_3d")
+
+
+def div_decompress_3d(desc: DivDesc3D, comp_ptr: int, comp_bytes: int, xhat_ptr: int, stream: int = 0) -> None:
+    _check(lib().div_decompress_3d(ctypes.byref(desc), c_void_p(comp_ptr), comp_bytes, c_void_p(xhat_ptr), c_void_p(stream)),
+           "div_decompress_3d")
 
 
 def div_mask_bytes(total: int) -> int:

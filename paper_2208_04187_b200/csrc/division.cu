@@ -17,6 +17,7 @@
 #include "planegroup.cuh"
 #include "planes.cuh"
 #include "twopass.cuh"
+#include "volume.cuh"
 
 namespace {
 
@@ -613,6 +614,134 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
                 if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
                 pg_decompress_general_kernel<XT, LT, Q><<<(unsigned)g, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, s, nwords);
             }
+            return launch_status();
+        });
+    });
+}
+
+// ------------------------------------------------------------------------------------------------
+// 3-D activation maps
+// ------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+div_status check_desc3(const div_desc3d* d) {
+    if (!d) return DIV_ERR_NULL;
+    if (d->n < 1 || d->c < 1 || d->d < 1 || d->h < 1 || d->w < 1) return DIV_ERR_SHAPE;
+    if (d->n >= (1ll << 31) || d->c >= (1ll << 32) || d->d >= (1ll << 32) || d->h >= (1ll << 32) || d->w >= (1ll << 32))
+        return DIV_ERR_SHAPE;
+    const unsigned __int128 per = (unsigned __int128)d->c * (unsigned __int128)d->d * (unsigned __int128)d->h * (unsigned __int128)d->w;
+    if (per >= ((unsigned __int128)1 << 32)) return DIV_ERR_SHAPE;
+    if (d->block < 1) return DIV_ERR_PARAM;
+    if (!(d->qbits == 1 || d->qbits == 2 || d->qbits == 4 || d->qbits == 8)) return DIV_ERR_PARAM;
+    if (!(d->x_dtype == DIV_F32 || d->x_dtype == DIV_BF16)) return DIV_ERR_PARAM;
+    if (!(d->lfc_dtype == DIV_F32 || d->lfc_dtype == DIV_BF16)) return DIV_ERR_PARAM;
+    return DIV_OK;
+}
+
+Shape3 make_shape3(const div_desc3d* d) {
+    Shape3 s;
+    s.N = (uint32_t)d->n;
+    s.C = (uint32_t)d->c;
+    s.D = (uint32_t)d->d;
+    s.H = (uint32_t)d->h;
+    s.W = (uint32_t)d->w;
+    uint32_t big = s.D > s.H ? s.D : s.H;
+    if (s.W > big) big = s.W;
+    s.B = (uint32_t)d->block > big ? big : (uint32_t)d->block;     // a block larger than every side is the largest side
+    s.Db = (s.D + s.B - 1) / s.B;
+    s.Hb = (s.H + s.B - 1) / s.B;
+    s.Wb = (s.W + s.B - 1) / s.B;
+    s.P2 = 1;
+    while (s.P2 < s.B) s.P2 <<= 1;
+    s.HW = s.H * s.W;
+    s.DHW = s.D * s.HW;
+    s.CDHW = s.C * s.DHW;
+    s.TPV = s.Db * s.Hb * s.Wb;
+    s.total = (uint64_t)s.N * s.CDHW;
+    s.tiles = (uint64_t)s.N * s.C * s.TPV;
+    return s;
+}
+
+void make_layout3(const div_desc3d* d, const Shape3& s, div_layout* out) {
+    out->lfc_off = 0;
+    out->lfc_bytes = s.tiles * dtype_bytes(d->lfc_dtype);
+    out->packed_off = align_up(out->lfc_bytes, SECTION_ALIGN);
+    out->packed_bytes = ((s.total * (uint64_t)d->qbits + 31) / 32) * 4;
+    out->stats_off = align_up(out->packed_off + out->packed_bytes, SECTION_ALIGN);
+    out->stats_bytes = 8ull * s.N;
+    out->total_bytes = out->stats_off + out->stats_bytes;
+    out->closed_form_bytes = out->lfc_bytes + out->packed_bytes + out->stats_bytes;
+    out->raw_bytes = s.total * dtype_bytes(d->x_dtype);
+    out->workspace_bytes = align_up(4ull * (WS_HEADER_WORDS + (uint64_t)WS_SLOT_WORDS * s.N), 256);
+}
+
+}  // namespace
+
+extern "C" {
+
+div_status div_compressed_bytes_3d(const div_desc3d* desc, div_layout* out) {
+    if (!desc || !out) return DIV_ERR_NULL;
+    const div_status st = check_desc3(desc);
+    if (st != DIV_OK) return st;
+    make_layout3(desc, make_shape3(desc), out);
+    return DIV_OK;
+}
+
+div_status div_compress_3d(const div_desc3d* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
+                           void* workspace_dev, size_t workspace_bytes, uint64_t seed, void* cuda_stream) {
+    if (!desc || !x_dev || !comp_dev || !workspace_dev) return DIV_ERR_NULL;
+    div_status st = check_desc3(desc);
+    if (st != DIV_OK) return st;
+    if (!aligned16(x_dev) || !aligned16(comp_dev) || !aligned16(workspace_dev)) return DIV_ERR_ALIGN;
+    const Shape3 s = make_shape3(desc);
+    div_layout lo;
+    make_layout3(desc, s, &lo);
+    if (comp_capacity < lo.total_bytes || workspace_bytes < lo.workspace_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
+    uint8_t* blob = (uint8_t*)comp_dev;
+    uint32_t* ws = (uint32_t*)workspace_dev;
+    const uint64_t nwords = lo.packed_bytes / 4;
+    const uint64_t g1 = (s.tiles + 127) / 128, g2 = (nwords + 255) / 256;
+    if (g1 > 0x7FFFFFFFull || g2 > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
+    return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        lfc_stats3d_kernel<XT, LT><<<(unsigned)g1, 128, 0, stream>>>((const XT*)x_dev, (LT*)(blob + lo.lfc_off), ws, s);
+        if (launch_status() != DIV_OK) return DIV_ERR_CUDA;
+        return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+            quant_pack3d_kernel<XT, LT, decltype(q)::value><<<(unsigned)g2, 256, 0, stream>>>(
+                (const XT*)x_dev, (const LT*)(blob + lo.lfc_off), ws, (uint32_t*)(blob + lo.packed_off),
+                (float*)(blob + lo.stats_off), s, seed, nwords);
+            return launch_status();
+        });
+    });
+}
+
+div_status div_decompress_3d(const div_desc3d* desc, const void* comp_dev, size_t comp_bytes, void* xhat_dev,
+                             void* cuda_stream) {
+    if (!desc || !comp_dev || !xhat_dev) return DIV_ERR_NULL;
+    div_status st = check_desc3(desc);
+    if (st != DIV_OK) return st;
+    if (!aligned16(comp_dev) || !aligned16(xhat_dev)) return DIV_ERR_ALIGN;
+    const Shape3 s = make_shape3(desc);
+    div_layout lo;
+    make_layout3(desc, s, &lo);
+    if (comp_bytes < lo.total_bytes) return DIV_ERR_CAPACITY;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const uint8_t* blob = (const uint8_t*)comp_dev;
+    const uint64_t nwords = lo.packed_bytes / 4;
+    const uint64_t g = (nwords + 255) / 256;
+    if (g > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
+    return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
+        typedef std::remove_pointer_t<decltype(xt)> XT;
+        typedef std::remove_pointer_t<decltype(lt)> LT;
+        return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+            decompress3d_kernel<XT, LT, decltype(q)::value><<<(unsigned)g, 256, 0, stream>>>(
+                (const LT*)(blob + lo.lfc_off), (const uint32_t*)(blob + lo.packed_off), (const float*)(blob + lo.stats_off),
+                (XT*)xhat_dev, s, nwords);
             return launch_status();
         });
     });

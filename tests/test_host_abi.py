@@ -20,7 +20,7 @@ def built_library():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "division.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(div_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(div_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_library_exports_every_declared_symbol():
@@ -75,6 +75,18 @@ def test_planegroup_refuses_too_many_planes_and_bad_flags():
     assert L.div_planegroup_compress(ctypes.byref(d), 16, 32, 8, 0, None, 0) == binding.DIV_ERR_CAPACITY
     assert L.div_planegroup_decompress(ctypes.byref(d), 16, 8, 32, None) == binding.DIV_ERR_CAPACITY
     assert L.div_planegroup_decompress(ctypes.byref(d), 16, 1 << 20, 34, None) == binding.DIV_ERR_ALIGN
+
+
+@pytest.mark.parametrize("d", [(2, 3, 8, 8, 8, 4, 2, "f32", "f32"), (3, 5, 8, 16, 24, 8, 2, "f32", "bf16"),
+                               (1, 2, 5, 9, 7, 4, 4, "bf16", "bf16"), (2, 2, 3, 3, 3, 8, 8, "f32", "f32"),
+                               (4, 7, 1, 14, 14, 8, 1, "f32", "f32")])
+def test_3d_bytes_match_the_closed_form(d):
+    m, c, dd, h, w, b, q, xd, ld = d
+    got = binding.div_compressed_bytes_3d(binding.make_desc_3d(*d))
+    ref = orc.layout_3d(m, c, dd, h, w, b, q, xd, ld)
+    for field in ("lfc_off", "lfc_bytes", "packed_off", "packed_bytes", "stats_off", "stats_bytes",
+                  "total_bytes", "closed_form_bytes", "raw_bytes"):
+        assert getattr(got, field) == getattr(ref, field), field
 
 
 def test_mask_bytes_and_host_checks():
