@@ -493,6 +493,45 @@ def run_ours(args):
                  "peak": t_peak, "peak_kind": f"of {t_peak_kind}", "gpu_launches": 9 * (t_steps + 3), "per_map": rows}
         del t_x, t_out, t_codec
 
+    # ---- one 3-D map (Minibatch x Channel x D x H x W; general kernels only) ----
+    three_d = None
+    if not args.no_one_d:
+        shp, b3, q3 = (8, 64, 16, 56, 56), 8, 2
+        desc3 = binding.make_desc_3d(*shp, b3, q3)
+        lo3 = binding.div_compressed_bytes_3d(desc3)
+        gen = torch.Generator(device=device).manual_seed(12)
+        pairs3 = [(torch.randn(*shp, device=device, generator=gen), torch.empty(shp, device=device)) for _ in range(2)]
+        blob3 = torch.empty(int(lo3.total_bytes), dtype=torch.uint8, device=device)
+        ws3 = torch.empty(int(lo3.workspace_bytes), dtype=torch.uint8, device=device)
+        stream = binding.current_stream_handle()
+        n3 = max(4, min(args.steps, 20))
+        ce3 = [(ev(), ev()) for _ in range(n3)]
+        de3 = [(ev(), ev()) for _ in range(n3)]
+        for k in range(-3, n3):
+            xin, xout = pairs3[k % 2]
+            if k >= 0:
+                ce3[k][0].record()
+            binding.div_compress_3d(desc3, xin.data_ptr(), blob3.data_ptr(), blob3.numel(), ws3.data_ptr(), ws3.numel(), 0, stream)
+            if k >= 0:
+                ce3[k][1].record()
+                de3[k][0].record()
+            binding.div_decompress_3d(desc3, blob3.data_ptr(), blob3.numel(), xout.data_ptr(), stream)
+            if k >= 0:
+                de3[k][1].record()
+        barrier()
+        c_us = statistics.mean(a.elapsed_time(b) for a, b in ce3) * 1e3
+        d_us = statistics.mean(a.elapsed_time(b) for a, b in de3) * 1e3
+        b3y = int(lo3.raw_bytes) + int(lo3.closed_form_bytes)
+        pk3, pk3_kind = measured_peak()
+        three_d = {"what": "3-D map " + "x".join(map(str, shp)) + f" fp32, B={b3}, Q={q3}; general kernels (one thread per block, one per packed word), this rank",
+                   "compression_ratio": int(lo3.raw_bytes) / int(lo3.closed_form_bytes), "steps": n3,
+                   "compress_kernel": "lfc_stats3d_kernel + quant_pack3d_kernel", "compress_us": round(c_us, 1),
+                   "compress_GBps": round(b3y / c_us / 1e3, 1), "compress_frac_of_peak": round(b3y / c_us / 1e3 / pk3, 3),
+                   "decompress_kernel": "decompress3d_kernel", "decompress_us": round(d_us, 1),
+                   "decompress_GBps": round(b3y / d_us / 1e3, 1), "decompress_frac_of_peak": round(b3y / d_us / 1e3 / pk3, 3),
+                   "peak_kind": f"of {pk3_kind}", "gpu_launches": 3 * (n3 + 3)}
+        del pairs3, blob3, ws3
+
     # ---- Algorithm 1 around a synthetic ResNet-50 step: activation memory (after forward - after backward) and
     # ---- forward+backward time, plain autograd against the cache (B=8, Q=2; ReLU with packed masks) ----
     train_step = None
@@ -558,6 +597,7 @@ def run_ours(args):
         "plane_groups": plane_groups,
         "mask_ops": mask_ops,
         "one_d": one_d,
+        "three_d": three_d,
         "train_step": train_step,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
@@ -579,7 +619,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-plane-groups", action="store_true", help="skip the extra timed loop of the per-plane form")
     ap.add_argument("--no-train-step", action="store_true", help="skip the ResNet-50 forward+backward memory / time measurement")
-    ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D maps")
+    ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D and 3-D maps")
     ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
     ap.add_argument("--compress-flags", type=int, default=0,
