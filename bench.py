@@ -493,7 +493,7 @@ def run_ours(args):
                  "peak": t_peak, "peak_kind": f"of {t_peak_kind}", "gpu_launches": 9 * (t_steps + 3), "per_map": rows}
         del t_x, t_out, t_codec
 
-    # ---- one 3-D map (Minibatch x Channel x D x H x W; general kernels only) ----
+    # ---- one 3-D map (Minibatch x Channel x D x H x W) ----
     three_d = None
     if not args.no_one_d:
         shp, b3, q3 = (8, 64, 16, 56, 56), 8, 2
@@ -523,11 +523,11 @@ def run_ours(args):
         d_us = statistics.mean(a.elapsed_time(b) for a, b in de3) * 1e3
         b3y = int(lo3.raw_bytes) + int(lo3.closed_form_bytes)
         pk3, pk3_kind = measured_peak()
-        three_d = {"what": "3-D map " + "x".join(map(str, shp)) + f" fp32, B={b3}, Q={q3}; general kernels (one thread per block, one per packed word), this rank",
+        three_d = {"what": "3-D map " + "x".join(map(str, shp)) + f" fp32, B={b3}, Q={q3}, this rank",
                    "compression_ratio": int(lo3.raw_bytes) / int(lo3.closed_form_bytes), "steps": n3,
-                   "compress_kernel": "lfc_stats3d_kernel + quant_pack3d_kernel", "compress_us": round(c_us, 1),
+                   "compress_kernel": "lfc_stats3d_warp_kernel + quant3d_quad_kernel", "compress_us": round(c_us, 1),
                    "compress_GBps": round(b3y / c_us / 1e3, 1), "compress_frac_of_peak": round(b3y / c_us / 1e3 / pk3, 3),
-                   "decompress_kernel": "decompress3d_kernel", "decompress_us": round(d_us, 1),
+                   "decompress_kernel": "decompress3d_quad_kernel", "decompress_us": round(d_us, 1),
                    "decompress_GBps": round(b3y / d_us / 1e3, 1), "decompress_frac_of_peak": round(b3y / d_us / 1e3 / pk3, 3),
                    "peak_kind": f"of {pk3_kind}", "gpu_launches": 3 * (n3 + 3)}
         del pairs3, blob3, ws3

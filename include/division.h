@@ -244,7 +244,8 @@ div_status div_planegroup_plan_query(const div_desc* desc, uint32_t flags, div_p
  * tree along the depth axis, then down the rows, then across the columns; in-sample index
  * e = ((c*D + d)*H + h)*W + w; one fp32 (delta, Delta) pair per sample; blob = [lfc: N*C*ceil(D/B)*ceil(H/B)*
  * ceil(W/B) values | packed | stats] with the same padding, workspace as for div_compress.  c*d*h*w < 2^32.
- * General kernels only (one thread per block, then one per packed word): any shape, block size and Q.
+ * Any shape, block size and Q; faster kernels where the padded block side is at most 32 (block means) and where
+ * W%4==0 and B%4==0 (quantise, decompress).
  * Arguments, ownership and error codes as for div_compressed_bytes / div_compress / div_decompress.
  */
 typedef struct div_desc3d {

@@ -664,6 +664,26 @@ Shape3 make_shape3(const div_desc3d* d) {
     return s;
 }
 
+// quad kernels of the 3-D form: 4 consecutive elements share a block
+bool quad3_ok(const Shape3& s) { return s.W % 4 == 0 && s.B % 4 == 0 && s.CDHW < (1u << 31) && s.N <= 65535; }
+Quad3 make_quad3(const Shape3& s) {
+    Quad3 g;
+    g.qps = s.CDHW / 4;
+    g.C = s.C;
+    g.Db = s.Db;
+    g.Hb = s.Hb;
+    g.Wb = s.Wb;
+    g.B = s.B;
+    g.qpr = s.W / 4;
+    g.qpp = s.H * g.qpr;
+    g.qpv = s.D * g.qpp;
+    g.by_qpv = make_fastdiv(g.qpv);
+    g.by_qpp = make_fastdiv(g.qpp);
+    g.by_qpr = make_fastdiv(g.qpr);
+    g.by_b = make_fastdiv(s.B);
+    return g;
+}
+
 void make_layout3(const div_desc3d* d, const Shape3& s, div_layout* out) {
     out->lfc_off = 0;
     out->lfc_bytes = s.tiles * dtype_bytes(d->lfc_dtype);
@@ -703,14 +723,50 @@ div_status div_compress_3d(const div_desc3d* desc, const void* x_dev, void* comp
     if (cudaMemsetAsync(workspace_dev, 0, lo.workspace_bytes, stream) != cudaSuccess) return DIV_ERR_CUDA;
     uint8_t* blob = (uint8_t*)comp_dev;
     uint32_t* ws = (uint32_t*)workspace_dev;
+    // kernels that store bytes or half-words leave the unused top of a partial last word alone: it is zero by contract
+    if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
+        cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
+        return DIV_ERR_CUDA;
     const uint64_t nwords = lo.packed_bytes / 4;
     const uint64_t g1 = (s.tiles + 127) / 128, g2 = (nwords + 255) / 256;
     if (g1 > 0x7FFFFFFFull || g2 > 0x7FFFFFFFull) return DIV_ERR_SHAPE;
     return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
         typedef std::remove_pointer_t<decltype(xt)> XT;
         typedef std::remove_pointer_t<decltype(lt)> LT;
-        lfc_stats3d_kernel<XT, LT><<<(unsigned)g1, 128, 0, stream>>>((const XT*)x_dev, (LT*)(blob + lo.lfc_off), ws, s);
+        // blocks whose padded side fits a warp: a lane per block column (coalesced); else a thread per block
+        const uint32_t bpw = s.P2 <= 32u ? 32u / s.P2 : 0u;
+        const uint32_t gpr = bpw ? (s.Wb + bpw - 1u) / bpw : 0u;                       // warp groups per row of blocks
+        const uint64_t groups = (uint64_t)s.N * s.C * s.Db * s.Hb * gpr;
+        const uint64_t gw = (groups + 7u) / 8u;
+        if (bpw && gw <= 0x7FFFFFFFull) {
+            const XT* xs = (const XT*)x_dev;
+            LT* lf = (LT*)(blob + lo.lfc_off);
+            switch (s.P2) {
+                case 1: lfc_stats3d_warp_kernel<XT, LT, 1><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+                case 2: lfc_stats3d_warp_kernel<XT, LT, 2><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+                case 4: lfc_stats3d_warp_kernel<XT, LT, 4><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+                case 8: lfc_stats3d_warp_kernel<XT, LT, 8><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+                case 16: lfc_stats3d_warp_kernel<XT, LT, 16><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+                default: lfc_stats3d_warp_kernel<XT, LT, 32><<<(unsigned)gw, 256, 0, stream>>>(xs, lf, ws, s, gpr, groups); break;
+            }
+        } else {
+            lfc_stats3d_kernel<XT, LT><<<(unsigned)g1, 128, 0, stream>>>((const XT*)x_dev, (LT*)(blob + lo.lfc_off), ws, s);
+        }
         if (launch_status() != DIV_OK) return DIV_ERR_CUDA;
+        if (quad3_ok(s) && desc->qbits != 1) {
+            const Quad3 g = make_quad3(s);
+            const dim3 grid((g.qps + 256u * DEC_QPT - 1) / (256u * DEC_QPT), s.N);
+            void* packed = blob + lo.packed_off;
+            float* stats = (float*)(blob + lo.stats_off);
+            const XT* xs = (const XT*)x_dev;
+            const LT* lf = (const LT*)(blob + lo.lfc_off);
+            switch (desc->qbits) {
+                case 2: quant3d_quad_kernel<XT, LT, 2, DEC_QPT><<<grid, 256, 0, stream>>>(xs, lf, ws, packed, stats, g, seed); break;
+                case 4: quant3d_quad_kernel<XT, LT, 4, DEC_QPT><<<grid, 256, 0, stream>>>(xs, lf, ws, packed, stats, g, seed); break;
+                default: quant3d_quad_kernel<XT, LT, 8, DEC_QPT><<<grid, 256, 0, stream>>>(xs, lf, ws, packed, stats, g, seed); break;
+            }
+            return launch_status();
+        }
         return dispatch_q(desc->qbits, [&](auto q) -> div_status {
             quant_pack3d_kernel<XT, LT, decltype(q)::value><<<(unsigned)g2, 256, 0, stream>>>(
                 (const XT*)x_dev, (const LT*)(blob + lo.lfc_off), ws, (uint32_t*)(blob + lo.packed_off),
@@ -738,6 +794,16 @@ div_status div_decompress_3d(const div_desc3d* desc, const void* comp_dev, size_
     return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
         typedef std::remove_pointer_t<decltype(xt)> XT;
         typedef std::remove_pointer_t<decltype(lt)> LT;
+        if (quad3_ok(s)) {
+            const Quad3 g3 = make_quad3(s);
+            const dim3 grid((g3.qps + 256u * DEC_QPT - 1) / (256u * DEC_QPT), s.N);
+            return dispatch_q(desc->qbits, [&](auto q) -> div_status {
+                decompress3d_quad_kernel<XT, LT, decltype(q)::value, DEC_QPT><<<grid, 256, 0, stream>>>(
+                    (const LT*)(blob + lo.lfc_off), (const uint32_t*)(blob + lo.packed_off), (const float*)(blob + lo.stats_off),
+                    (XT*)xhat_dev, g3);
+                return launch_status();
+            });
+        }
         return dispatch_q(desc->qbits, [&](auto q) -> div_status {
             decompress3d_kernel<XT, LT, decltype(q)::value><<<(unsigned)g, 256, 0, stream>>>(
                 (const LT*)(blob + lo.lfc_off), (const uint32_t*)(blob + lo.packed_off), (const float*)(blob + lo.stats_off),

@@ -4,13 +4,15 @@
 //   lfc_stats3d_kernel   one thread per block: mean in the fixed order (balanced pairwise tree along the depth
 //                        axis, then down the rows, then across the columns), stored low-frequency value,
 //                        residual extremes -> per-sample min / max keys in the scratch slots
+//   lfc_stats3d_warp_kernel  the same with a lane per block column (blocks of padded side <= 32): coalesced loads
 //   quant_pack3d_kernel  one thread per packed 32-bit word
 //   decompress3d_kernel  one thread per packed 32-bit word
 // x is read twice by compress (the second time from L2 when the tensor fits).
 #pragma once
 
-#include "common.cuh"
-#include "twopass.cuh"   // tree_sum
+#include "decompress.cuh"   // DeqTable, quad_bits, Quad
+#include "fused_v.cuh"     // packed arithmetic, quant_row
+#include "twopass.cuh"     // tree_sum
 
 namespace divk {
 
@@ -57,6 +59,64 @@ lfc_stats3d_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
     uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
     atomicMax(slot + 0, ~float_key(__fsub_rn(lo, stored)));
     atomicMax(slot + 1, float_key(__fsub_rn(hi, stored)));
+}
+
+// The same for blocks whose padded side fits a warp (P2 <= 32): a lane owns one column of one block, the P2 lanes
+// of a block sit side by side and a warp takes 32 / P2 blocks that are neighbours along w, so every load
+// instruction of a warp reads one contiguous row segment.  A lane sums its column along the depth and down the
+// rows (the same trees), the columns of a block meet through xor shuffles.  One warp per group of 32 / P2 blocks.
+template <typename XT, typename LT, int P2>
+__global__ void __launch_bounds__(256)
+lfc_stats3d_warp_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, Shape3 s,
+                        uint32_t groups_per_row, uint64_t groups) {
+    constexpr uint32_t BPW = 32 / P2;                         // blocks per warp
+    const uint64_t grp = (uint64_t)blockIdx.x * 8u + (threadIdx.x >> 5);
+    if (grp >= groups) return;                                // whole warps leave together
+    const uint32_t lane = threadIdx.x & 31;
+    // group -> (volume, bd, bh, first bw)
+    const uint64_t rowid = grp / groups_per_row;              // (vol * Db + bd) * Hb + bh
+    const uint32_t bw = (uint32_t)(grp - rowid * groups_per_row) * BPW + lane / P2;
+    const uint32_t cw = lane % P2;
+    const uint64_t vd = rowid / s.Hb;
+    const uint32_t bh = (uint32_t)(rowid - vd * s.Hb);
+    const uint64_t vol = vd / s.Db;
+    const uint32_t bd = (uint32_t)(vd - vol * s.Db);
+    const uint32_t n = (uint32_t)(vol / s.C);
+    const uint32_t d0 = bd * s.B, h0 = bh * s.B, w0 = bw * s.B;
+    const uint32_t nd = min(s.B, s.D - d0), nh = min(s.B, s.H - h0);
+    const uint32_t nw = bw < s.Wb ? min(s.B, s.W - w0) : 0u;
+    const bool ok = cw < nw;
+    const XT* base = x + vol * s.DHW + ((size_t)d0 * s.H + h0) * s.W + (ok ? w0 + cw : 0u);
+    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+    float sum = tree_sum((uint32_t)P2, [&](uint32_t r) -> float {
+        if (!ok || r >= nh) return 0.f;
+        return tree_sum((uint32_t)P2, [&](uint32_t k) -> float {
+            if (k >= nd) return 0.f;
+            const float v = Elem<XT>::load(base + ((size_t)k * s.H + r) * s.W);
+            lo = fminf(lo, v);
+            hi = fmaxf(hi, v);
+            return v;
+        });
+    });
+#pragma unroll
+    for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+    uint32_t kmin = 0u, kmax = 0u;                            // neutral keys
+    if (bw < s.Wb) {
+        const float mean = __fdiv_rn(sum, (float)(nd * nh * nw));
+        const float stored = Elem<LT>::round(mean);
+        if (cw == 0) Elem<LT>::store(lfc + ((vol * s.Db + bd) * s.Hb + bh) * s.Wb + bw, mean);
+        if (ok) {
+            kmin = ~float_key(__fsub_rn(lo, stored));         // x -> fl(x - stored) is monotone
+            kmax = float_key(__fsub_rn(hi, stored));
+        }
+    }
+    kmin = __reduce_max_sync(0xFFFFFFFFu, kmin);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+    if (lane == 0) {
+        uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+        atomicMax(slot + 0, kmin);
+        atomicMax(slot + 1, kmax);
+    }
 }
 
 // position of a flat in-sample index
@@ -157,6 +217,96 @@ decompress3d_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ pac
         }
         Elem<XT>::store(xhat + i, reconstruct((bits >> (j * Q)) & MASK, step, delta, Elem<LT>::load(lfc + lfc_index3(s, n, p))));
         advance3(s, n, e, p);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// W % 4 == 0 and B % 4 == 0: 4 consecutive elements share a block.  One thread per QPT quads, 256 quads apart.
+// grid = (ceil(quads_per_sample / (256*QPT)), N)
+// ------------------------------------------------------------------------------------------------
+struct Quad3 {
+    uint32_t qps;                 // quads per sample
+    uint32_t C, Db, Hb, Wb, B;
+    uint32_t qpr, qpp, qpv;       // quads per row, per plane (H rows), per volume (D planes)
+    FastDiv by_qpv, by_qpp, by_qpr, by_b;
+};
+// low-frequency value of quad q (inside sample n's map lfc_n)
+template <typename LT>
+__device__ __forceinline__ float quad3_lfc(const LT* __restrict__ lfc_n, const Quad3& g, uint32_t q) {
+    const uint32_t vol = fdiv(q, g.by_qpv);
+    uint32_t rem = q - vol * g.qpv;
+    const uint32_t d = fdiv(rem, g.by_qpp);
+    rem -= d * g.qpp;
+    const uint32_t h = fdiv(rem, g.by_qpr);
+    const uint32_t w = (rem - h * g.qpr) * 4u;
+    return Elem<LT>::load(lfc_n + (((size_t)vol * g.Db + fdiv(d, g.by_b)) * g.Hb + fdiv(h, g.by_b)) * g.Wb + fdiv(w, g.by_b));
+}
+
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+quant3d_quad_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const uint32_t* __restrict__ ws,
+                    void* __restrict__ packed_v, float* __restrict__ stats, Quad3 g, uint64_t seed) {
+    typedef typename PackedUnit<Q>::type OutT;
+    const uint32_t n = blockIdx.y;
+    const uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+    const QParams qp = make_qparams(key_float(~__ldg(slot + 0)), key_float(__ldg(slot + 1)), Q);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        stats[2 * (size_t)n + 0] = qp.delta;
+        stats[2 * (size_t)n + 1] = qp.step;
+    }
+    const uint64_t delta2 = pk2(qp.delta, qp.delta), scale2 = pk2(qp.scale, qp.scale);
+    const uint64_t base = rng_sample_base(seed, n);
+    const XT* x_n = x + (size_t)n * g.qps * 4u;
+    const LT* lfc_n = lfc + (size_t)n * g.C * g.Db * g.Hb * g.Wb;
+    OutT* packed = reinterpret_cast<OutT*>(packed_v) + (uint64_t)n * g.qps;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint64_t xy[QPT], zw[QPT];
+    float lf[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < g.qps) {
+            StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy[k], zw[k]);
+            lf[k] = quad3_lfc(lfc_n, g, q);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < g.qps)
+            packed[q] = (OutT)quant_row<Q>(xy[k], zw[k], pk2(lf[k], lf[k]), delta2, scale2, rng_group(base, q));
+    }
+}
+
+template <typename XT, typename LT, int Q, int QPT>
+__global__ void __launch_bounds__(256)
+decompress3d_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
+                         const float* __restrict__ stats, XT* __restrict__ xhat, Quad3 g) {
+    __shared__ DeqTable<Q> table;
+    const uint32_t n = blockIdx.y;
+    table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
+    __syncthreads();
+    const uint64_t sample_quad0 = (uint64_t)n * g.qps;
+    const LT* lfc_n = lfc + (size_t)n * g.C * g.Db * g.Hb * g.Wb;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint32_t bits[QPT];
+    float lf[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < g.qps) {
+            bits[k] = quad_bits<Q>(packed, sample_quad0 + q);
+            lf[k] = quad3_lfc(lfc_n, g, q);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        if (q < g.qps) {
+            const float4 hq = table.quad(bits[k]);
+            Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, __fadd_rn(lf[k], hq.x), __fadd_rn(lf[k], hq.y),
+                            __fadd_rn(lf[k], hq.z), __fadd_rn(lf[k], hq.w));
+        }
     }
 }
 

@@ -28,8 +28,9 @@ def run(x, block, q, seed, xd, ld):
     lo = binding.div_compressed_bytes_3d(desc)
     t = torch.from_numpy(x)
     xdev = (t.view(torch.bfloat16) if xd == "bf16" else t).cuda()
-    blob = torch.full((int(lo.total_bytes) + 64,), 0x5A, dtype=torch.uint8, device="cuda")
-    blob[:int(lo.total_bytes)] = 0
+    blob = torch.full((int(lo.total_bytes) + 64,), 0x5A, dtype=torch.uint8, device="cuda")   # stale bytes everywhere ...
+    blob[int(lo.lfc_bytes):int(lo.packed_off)] = 0                                          # ... but in the padding,
+    blob[int(lo.packed_off + lo.packed_bytes):int(lo.stats_off)] = 0                        # which is never written
     ws = torch.empty(int(lo.workspace_bytes), dtype=torch.uint8, device="cuda")
     out = torch.empty_like(xdev)
     s = torch.cuda.current_stream().cuda_stream
@@ -45,6 +46,8 @@ CASES = [
     ((2, 2, 3, 3, 3), 8, 8, "bf16", "bf16"), ((3, 2, 6, 10, 4), 3, 1, "f32", "f32"), ((2, 5, 1, 14, 14), 8, 2, "f32", "f32"),
     ((2, 4, 2, 12, 20), 8, 2, "bf16", "f32"), ((1, 1, 1, 1, 1), 8, 2, "f32", "f32"), ((3, 3, 7, 5, 3), 2, 2, "f32", "f32"),
     ((2, 8, 16, 28, 28), 8, 2, "f32", "f32"), ((2, 3, 4, 4, 33), 16, 4, "f32", "f32"),
+    ((1, 3, 1, 3, 4), 4, 2, "f32", "f32"), ((2, 5, 6, 10, 24), 12, 4, "bf16", "bf16"), ((2, 4, 9, 8, 16), 16, 8, "f32", "f32"),
+    ((3, 2, 5, 7, 12), 4, 1, "f32", "f32"), ((1, 2, 40, 12, 8), 8, 2, "f32", "bf16"),
 ]
 
 
