@@ -269,7 +269,12 @@ def torch_dtype(name: str):
 
 
 def current_stream_handle() -> int:
-    return int(_torch().cuda.current_stream().cuda_stream)
+    """cudaStream_t of torch's current stream on the current device, as an integer."""
+    torch = _torch()
+    raw = getattr(torch._C, "_cuda_getCurrentRawStream", None)      # one C call instead of building a Stream object
+    if raw is not None:
+        return int(raw(torch.cuda.current_device()))
+    return int(torch.cuda.current_stream().cuda_stream)
 
 
 class Codec:
