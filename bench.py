@@ -300,23 +300,30 @@ def run_ours(args):
         assert c.device_status() == binding.DIV_OK
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    records = [[[(ev(), ev()) for _ in codecs] for _ in range(2)] for _ in range(args.steps)]
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.25)
     barrier()
+    # the timed region: exactly args.steps steps between two events, nothing else on the stream
     t_start, t_end = ev(), ev()
     t_start.record()
     for k in range(args.steps):
-        step(records[k])
+        step()
     t_end.record()
     barrier()
-    clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
+    # a second, instrumented pass for the per-call figures (an event pair around every call costs a few us per
+    # call, which is why it is kept out of the timed region above)
+    rec_steps = max(3, min(args.steps, 100))
+    records = [[[(ev(), ev()) for _ in codecs] for _ in range(2)] for _ in range(rec_steps)]
+    for k in range(rec_steps):
+        step(records[k])
+    barrier()
+    clocks = sampler.stop()
 
-    comp_ms = [statistics.mean(records[k][0][i][0].elapsed_time(records[k][0][i][1]) for k in range(args.steps))
+    comp_ms = [statistics.mean(records[k][0][i][0].elapsed_time(records[k][0][i][1]) for k in range(rec_steps))
                for i in range(len(codecs))]
-    dec_ms = [statistics.mean(records[k][1][i][0].elapsed_time(records[k][1][i][1]) for k in range(args.steps))
+    dec_ms = [statistics.mean(records[k][1][i][0].elapsed_time(records[k][1][i][1]) for k in range(rec_steps))
               for i in range(len(codecs))]
 
     # ---- end to end through the C ABI with host buffers: H2D of x, compress, decompress, D2H of x_hat ----
@@ -364,14 +371,17 @@ def run_ours(args):
         for _ in range(3):
             pg_step()
         barrier()
-        pg_rec = [[[(ev(), ev()) for _ in pg] for _ in range(2)] for _ in range(pg_steps)]
         p0, p1 = ev(), ev()
         p0.record()
         for k in range(pg_steps):
-            pg_step(pg_rec[k])
+            pg_step()
         p1.record()
         barrier()
         pg_ms = p0.elapsed_time(p1) / pg_steps
+        pg_rec = [[[(ev(), ev()) for _ in pg] for _ in range(2)] for _ in range(pg_steps)]
+        for k in range(pg_steps):
+            pg_step(pg_rec[k])
+        barrier()
         pg_comp = [statistics.mean(pg_rec[k][0][i][0].elapsed_time(pg_rec[k][0][i][1]) for k in range(pg_steps))
                    for i in range(len(pg))]
         pg_dec = [statistics.mean(pg_rec[k][1][i][0].elapsed_time(pg_rec[k][1][i][1]) for k in range(pg_steps))
@@ -468,14 +478,17 @@ def run_ours(args):
         for _ in range(3):
             t_step()
         barrier()
-        t_rec = [[[(ev(), ev()) for _ in t_codec] for _ in range(2)] for _ in range(t_steps)]
         q0, q1 = ev(), ev()
         q0.record()
         for k in range(t_steps):
-            t_step(t_rec[k])
+            t_step()
         q1.record()
         barrier()
         t_ms = q0.elapsed_time(q1) / t_steps
+        t_rec = [[[(ev(), ev()) for _ in t_codec] for _ in range(2)] for _ in range(t_steps)]
+        for k in range(t_steps):
+            t_step(t_rec[k])
+        barrier()
         t_raw = sum(int(c.layout.raw_bytes) for c in t_codec)
         t_peak, t_peak_kind = measured_peak()
         rows = []
@@ -582,10 +595,12 @@ def run_ours(args):
         "config": {"workload": WORKLOAD + (f" [maps {args.maps} only]" if args.maps else ""), "maps": [m["map"] for m in per_map],
                    "l2": "working set 1.2 GB per step, every buffer touched once per step: far above the 126 MB L2",
                    "order": "compress maps 0..4, then decompress maps 0..4",
+                   "timing": f"value / ms_per_step: {args.steps} steps between two CUDA events, nothing else on the stream; "
+                             f"per_map and roofline: a second pass of {rec_steps} steps with an event pair around every call",
                    "multi_gpu": "replicas only: each rank runs the same set on its own GPU, no collective",
                    "compression_ratio": raw_bytes / comp_bytes, "per_map": per_map},
         "roofline": {"bound": "hbm", "kernel": kernel_names[int(plans[dom].fused)] + " on " + per_map[dom]["map"] +
-                     " (CUDA events around the call on its stream; the span includes the 2-us workspace clear)",
+                     " (CUDA events around the call on its stream, instrumented pass; the span includes the 2-us workspace clear)",
                      "achieved": dom_gbs, "peak": peak, "unit": "GB/s", "frac": dom_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": dom_gbs / NOMINAL_HBM_GBS,
                      "traffic": NCU_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": algo_bytes[dom]},
