@@ -330,19 +330,44 @@ def run_ours(args):
     host_out = [torch.empty_like(h).pin_memory() for h in host_x]
     e2e_steps = max(2, min(args.steps, 5))
 
-    def e2e_step():
+    # three streams, so that the two PCIe directions and the kernels overlap: copy-in -> (compress, decompress) -> copy-out
+    # per map, each stage ordered after its predecessor by events; a buffer is reused only after its last reader is done
+    s_main = torch.cuda.current_stream(device)
+    s_in, s_out = torch.cuda.Stream(device), torch.cuda.Stream(device)
+    ev_in = [torch.cuda.Event() for _ in codecs]       # x[i] has arrived on the device
+    ev_done = [torch.cuda.Event() for _ in codecs]     # compress + decompress of map i have run (x[i] may be overwritten)
+    ev_out = [torch.cuda.Event() for _ in codecs]      # x_hat[i] has reached the host (dev_out[i] may be overwritten)
+
+    def e2e_step(first=False):
         for i, c in enumerate(codecs):
-            dev_x[i].copy_(host_x[i], non_blocking=True)
+            with torch.cuda.stream(s_in):
+                if not first:
+                    s_in.wait_event(ev_done[i])
+                dev_x[i].copy_(host_x[i], non_blocking=True)
+                ev_in[i].record(s_in)
+            s_main.wait_event(ev_in[i])
+            if not first:
+                s_main.wait_event(ev_out[i])
             c.compress(dev_x[i], seed=0, flags=args.compress_flags)
             c.decompress(out=dev_out[i])
-            host_out[i].copy_(dev_out[i], non_blocking=True)
+            ev_done[i].record(s_main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[i])
+                host_out[i].copy_(dev_out[i], non_blocking=True)
+                ev_out[i].record(s_out)
 
-    e2e_step()
+    def e2e_join():
+        for e in ev_out:
+            s_main.wait_event(e)
+
+    e2e_step(first=True)
+    e2e_join()
     barrier()
     e0, e1 = ev(), ev()
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
+    e2e_join()
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
@@ -616,7 +641,9 @@ def run_ours(args):
         "train_step": train_step,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
-                "steps": e2e_steps},
+                "steps": e2e_steps,
+                "how": "pinned host buffers; per map: copy-in, compress, decompress, copy-out, on three streams ordered by "
+                       "events so that the two PCIe directions and the kernels overlap"},
         "gpu_launches": kernels_per_step * args.steps,
         "clocks": clocks,
     }
