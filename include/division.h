@@ -92,9 +92,10 @@ typedef struct div_layout {
 /* How div_compress will run a descriptor (introspection for tests and benchmarks). */
 typedef struct div_plan {
     int32_t fused;          /* for W%4==0, B in {4,8}, Q in {2,4,8}, one launch:
+                               6: x read from HBM once and re-read from L2 a little later, both reads staged through
+                                  shared-memory rings by bulk copies (staged kernel; first choice from 40 MB up);
                                2: chunks wait in a shared-memory ring (strip ring kernel; first choice below 40 MB);
-                               3: x read from HBM once and re-read from L2 a little later (lagged kernel; first
-                                  choice from 40 MB up, and whenever the ring cannot hold a sample's share);
+                               3: as 6, with plain global loads (lagged kernel; next in line after 6 and 2);
                                4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
                                   at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;
@@ -120,6 +121,7 @@ typedef struct div_plan {
 #define DIV_FLAG_NO_LAGGED_KERNEL 4u /* never take the lagged (L2 re-read) kernel          */
 #define DIV_FLAG_NO_PLANE_KERNELS 8u /* never take the small-plane pair of kernels          */
 #define DIV_FLAG_NO_LINE_KERNELS 16u /* never take the pair of kernels for 1-D maps          */
+#define DIV_FLAG_NO_STAGED_KERNEL 32u/* never take the staged (bulk-copy rings) kernel       */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:
@@ -196,11 +198,12 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                           void* xhat_dev, void* cuda_stream);
 
 /*
- * Test hook for the bounded waits of the single-launch compress kernels (plan codes 2 and 3): runs the
+ * Test hook for the bounded waits of the single-launch compress kernels (plan codes 2, 3 and 6): runs the
  * kernel div_compress_ex would run, but tells it to wait for a number of arrivals per sample that is never
  * reached, with `timeout_ns` (at most 100 ms) as the limit of every wait.  The kernel must give up, record
  * DIV_ERR_TIMEOUT in the workspace status word (read it with div_read_device_status) and return; the blob's
- * contents are then unspecified.  Returns DIV_ERR_PARAM when the descriptor maps to neither kernel.
+ * contents are then unspecified.  The first of the strip ring, lagged and staged kernels that the flags allow
+ * and the descriptor fits is taken; DIV_ERR_PARAM when there is none.
  * Arguments as for div_compress_ex.  No counterpart in the paper.
  */
 div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,

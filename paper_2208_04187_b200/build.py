@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libdivision.so")
 SOURCES = ["division.cu"]
-HEADERS = ["common.cuh", "twopass.cuh", "decompress.cuh", "fused.cuh", "fused_v.cuh", "lagged.cuh", "planes.cuh", "planegroup.cuh", "masks.cuh", "lines.cuh", "volume.cuh", os.path.join("..", "..", "include", "division.h")]
+HEADERS = ["common.cuh", "twopass.cuh", "decompress.cuh", "fused.cuh", "fused_v.cuh", "lagged.cuh", "staged.cuh", "planes.cuh", "planegroup.cuh", "masks.cuh", "lines.cuh", "volume.cuh", os.path.join("..", "..", "include", "division.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

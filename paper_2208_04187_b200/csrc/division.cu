@@ -16,6 +16,7 @@
 #include "masks.cuh"
 #include "planegroup.cuh"
 #include "planes.cuh"
+#include "staged.cuh"
 #include "twopass.cuh"
 #include "volume.cuh"
 
@@ -26,7 +27,7 @@ typedef __nv_bfloat16 bf16;
 
 constexpr uint64_t SECTION_ALIGN = 128;
 constexpr uint32_t DIV_FLAG_ALL = DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL |
-                                  DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_NO_LINE_KERNELS;
+                                  DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_NO_LINE_KERNELS | DIV_FLAG_NO_STAGED_KERNEL;
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
@@ -158,10 +159,60 @@ div_status compress_two_pass(const div_desc* d, const Shape& s, const div_layout
 // ------------------------------------------------------------------------------------------
 constexpr int DEC_QPT = 4;
 
-// Large maps go to the lagged kernel first (measured: a few per cent faster from about 40 MB up), small ones
-// to the strip ring kernel (shorter start-up).
-bool prefer_lagged(const div_desc* d, const Shape& s) {
+// Which compress kernels run a descriptor.  Large maps go to the staged kernel (both reads of x staged through
+// shared memory by bulk copies), small ones to the strip ring kernel (shorter start-up); the lagged kernel
+// and the general kernels take what those two cannot.
+bool prefer_staged(const div_desc* d, const Shape& s) {
     return s.total * dtype_bytes(d->x_dtype) >= (40ull << 20);
+}
+
+struct Choice {
+    int code;          // the value div_plan.fused reports
+    LineGeom lg;
+    SPlan sp;
+    LPlan lp;
+    VPlan vp;
+    PlaneGeom pg;
+    FusedPlan fp;
+};
+
+void choose_compress(const div_desc* d, const Shape& s, uint32_t flags, Choice* c) {
+    const bool two_pass = (flags & DIV_FLAG_FORCE_TWO_PASS) != 0;
+    c->code = 0;
+    if (two_pass) return;
+    if (!(flags & DIV_FLAG_NO_LINE_KERNELS) && plan_lines(d, s, &c->lg)) {
+        c->code = 5;
+        return;
+    }
+    const bool may_staged = !(flags & DIV_FLAG_NO_STAGED_KERNEL);
+    const bool may_lag = !(flags & DIV_FLAG_NO_LAGGED_KERNEL);
+    const bool may_strip = !(flags & DIV_FLAG_NO_STRIP_KERNEL);
+    const bool big = prefer_staged(d, s);
+    if (may_staged && big && plan_staged(d, s, &c->sp) == DIV_OK) {
+        c->code = 6;
+        return;
+    }
+    if (may_lag && big && plan_lagged(d, s, &c->lp) == DIV_OK) {
+        c->code = 3;
+        return;
+    }
+    if (may_strip && plan_v(d, s, &c->vp) == DIV_OK) {
+        c->code = 2;
+        return;
+    }
+    if (may_lag && plan_lagged(d, s, &c->lp) == DIV_OK) {
+        c->code = 3;
+        return;
+    }
+    if (may_staged && plan_staged(d, s, &c->sp) == DIV_OK) {
+        c->code = 6;
+        return;
+    }
+    if (!(flags & DIV_FLAG_NO_PLANE_KERNELS) && plan_planes(d, s, &c->pg)) {
+        c->code = 4;
+        return;
+    }
+    if (plan_fused(d, s, &c->fp) == DIV_OK) c->code = 1;
 }
 
 bool decompress_fast_ok(const Shape& s) {
@@ -205,52 +256,49 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     if (flags & ~DIV_FLAG_ALL) return DIV_ERR_PARAM;
     const Shape s = make_shape(desc);
     *out = div_plan();
-    FusedPlan fp;
-    VPlan vp;
-    LPlan lp;
-    LineGeom lg;
-    const bool lines = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LINE_KERNELS)) && plan_lines(desc, s, &lg);
-    const bool lag_first = prefer_lagged(desc, s);
-    const bool lag_ok = !lines && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL)) && plan_lagged(desc, s, &lp) == DIV_OK;
-    const bool vec_ok = !lines && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL)) && plan_v(desc, s, &vp) == DIV_OK;
-    const bool lag = lag_ok && (lag_first || !vec_ok);
-    const bool vec = vec_ok && !lag;
-    PlaneGeom pg;
-    const bool planes = !lines && !lag && !vec && !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS)) && plan_planes(desc, s, &pg);
-    const bool fused = !lines && !lag && !vec && !planes && !(flags & DIV_FLAG_FORCE_TWO_PASS) && plan_fused(desc, s, &fp) == DIV_OK;
-    out->fused = lines ? 5 : (lag ? 3 : (vec ? 2 : (planes ? 4 : (fused ? 1 : 0))));
-    if (lines) {
-        out->grid = (int32_t)((lg.qps + 256 * LINE_QPT - 1) / (256 * LINE_QPT) * s.N);
+    Choice ch;
+    choose_compress(desc, s, flags, &ch);
+    out->fused = ch.code;
+    if (ch.code == 5) {
+        out->grid = (int32_t)((ch.lg.qps + 256 * LINE_QPT - 1) / (256 * LINE_QPT) * s.N);
         out->threads = 256;
         out->chunk_elems = 4 * LINE_QPT * 256;
-    } else if (lag) {
-        out->grid = lp.grid;
-        out->threads = lp.threads;
+    } else if (ch.code == 6) {
+        out->grid = ch.sp.grid;
+        out->threads = ch.sp.threads;
+        out->stages = (int32_t)(ch.sp.kr + ch.sp.kq);
+        out->lag = (int32_t)ch.sp.lag_chunks;
+        out->smem_bytes = ch.sp.smem_bytes;
+        out->chunk_elems = ch.sp.chunk_elems;
+        out->chunks_per_sample = ch.sp.chunks_per_sample;
+    } else if (ch.code == 3) {
+        out->grid = ch.lp.grid;
+        out->threads = ch.lp.threads;
         out->stages = 0;
-        out->lag = (int32_t)lp.lag_units;
+        out->lag = (int32_t)ch.lp.lag_units;
         out->smem_bytes = 0;
-        out->chunk_elems = (int64_t)32 * lp.bands_per_lane * 4 * s.B;       // elements of one full unit
-        out->chunks_per_sample = lp.units_per_sample;
-    } else if (vec) {
-        out->grid = vp.grid;
-        out->threads = vp.threads;
-        out->stages = vp.stages;
-        out->lag = vp.lag;
-        out->smem_bytes = vp.smem_bytes;
-        out->chunk_elems = vp.chunk_elems;
-        out->chunks_per_sample = vp.chunks_per_sample;
-    } else if (planes) {
-        out->grid = (int32_t)((pg.qps + 256 * PLANE_QPT - 1) / (256 * PLANE_QPT) * s.N);
+        out->chunk_elems = (int64_t)32 * ch.lp.bands_per_lane * 4 * s.B;       // elements of one full unit
+        out->chunks_per_sample = ch.lp.units_per_sample;
+    } else if (ch.code == 2) {
+        out->grid = ch.vp.grid;
+        out->threads = ch.vp.threads;
+        out->stages = ch.vp.stages;
+        out->lag = ch.vp.lag;
+        out->smem_bytes = ch.vp.smem_bytes;
+        out->chunk_elems = ch.vp.chunk_elems;
+        out->chunks_per_sample = ch.vp.chunks_per_sample;
+    } else if (ch.code == 4) {
+        out->grid = (int32_t)((ch.pg.qps + 256 * PLANE_QPT - 1) / (256 * PLANE_QPT) * s.N);
         out->threads = 256;
         out->chunk_elems = 4 * PLANE_QPT * 256;
-    } else if (fused) {
-        out->grid = fp.grid;
-        out->threads = fp.threads;
-        out->stages = fp.stages;
-        out->lag = fp.lag;
-        out->smem_bytes = fp.smem_bytes;
-        out->chunk_elems = fp.chunk_elems;
-        out->chunks_per_sample = fp.chunks_per_sample;
+    } else if (ch.code == 1) {
+        out->grid = ch.fp.grid;
+        out->threads = ch.fp.threads;
+        out->stages = ch.fp.stages;
+        out->lag = ch.fp.lag;
+        out->smem_bytes = ch.fp.smem_bytes;
+        out->chunk_elems = ch.fp.chunk_elems;
+        out->chunks_per_sample = ch.fp.chunks_per_sample;
     } else {
         out->grid = (int32_t)((s.tiles + 255) / 256);
         out->threads = 256;
@@ -279,27 +327,16 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
         cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
         return DIV_ERR_CUDA;
-    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LINE_KERNELS))) {
-        LineGeom lg;
-        if (plan_lines(desc, s, &lg)) return compress_lines(desc, s, lo, lg, x_dev, blob, ws, seed, stream);
-    }
-    const bool may_lag = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_LAGGED_KERNEL));
-    const bool may_strip = !(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL));
-    LPlan lp;
-    if (may_lag && prefer_lagged(desc, s) && plan_lagged(desc, s, &lp) == DIV_OK)
-        return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
-    if (may_strip) {
-        VPlan vp;
-        if (plan_v(desc, s, &vp) == DIV_OK) return compress_fused_v(desc, s, lo, vp, x_dev, blob, ws, seed, stream);
-    }
-    if (may_lag && plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream);
-    if (!(flags & (DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_PLANE_KERNELS))) {
-        PlaneGeom pg;
-        if (plan_planes(desc, s, &pg)) return compress_planes(desc, s, lo, pg, x_dev, blob, ws, seed, stream);
-    }
-    if (!(flags & DIV_FLAG_FORCE_TWO_PASS)) {
-        FusedPlan fp;
-        if (plan_fused(desc, s, &fp) == DIV_OK) return compress_fused(desc, s, lo, fp, x_dev, blob, ws, seed, stream);
+    Choice ch;
+    choose_compress(desc, s, flags, &ch);
+    switch (ch.code) {
+        case 5: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream);
+        case 6: return compress_staged(desc, s, lo, ch.sp, x_dev, blob, ws, seed, stream);
+        case 3: return compress_lagged(desc, s, lo, ch.lp, x_dev, blob, ws, seed, stream);
+        case 2: return compress_fused_v(desc, s, lo, ch.vp, x_dev, blob, ws, seed, stream);
+        case 4: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream);
+        case 1: return compress_fused(desc, s, lo, ch.fp, x_dev, blob, ws, seed, stream);
+        default: break;
     }
     return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
 }
@@ -328,6 +365,10 @@ div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, v
     if (!(flags & DIV_FLAG_NO_LAGGED_KERNEL)) {
         LPlan lp;
         if (plan_lagged(desc, s, &lp) == DIV_OK) return compress_lagged(desc, s, lo, lp, x_dev, blob, ws, seed, stream, never, timeout_ns);
+    }
+    if (!(flags & DIV_FLAG_NO_STAGED_KERNEL)) {
+        SPlan sp;
+        if (plan_staged(desc, s, &sp) == DIV_OK) return compress_staged(desc, s, lo, sp, x_dev, blob, ws, seed, stream, never, timeout_ns);
     }
     return DIV_ERR_PARAM;
 }

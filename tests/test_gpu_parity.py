@@ -16,10 +16,12 @@ from paper_2208_04187_b200 import binding, build, synth
 pytestmark = pytest.mark.gpu
 
 TWO_PASS = binding.DIV_FLAG_FORCE_TWO_PASS
-LAGGED = binding.DIV_FLAG_NO_STRIP_KERNEL          # skip the strip ring kernel: the lagged kernel is next in line
-RING = binding.DIV_FLAG_NO_LAGGED_KERNEL           # skip the lagged kernel: the strip ring kernel where it applies
-NO_STRIP = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL | binding.DIV_FLAG_NO_PLANE_KERNELS
-NO_SPECIAL = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL      # planes pair, else general ring
+# the three single-launch kernels for W % 4 == 0: each flag set leaves exactly one of them in line
+LAGGED = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_STAGED_KERNEL
+RING = binding.DIV_FLAG_NO_LAGGED_KERNEL | binding.DIV_FLAG_NO_STAGED_KERNEL
+STAGED = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL
+NO_SPECIAL = STAGED | binding.DIV_FLAG_NO_STAGED_KERNEL                     # planes pair, else general ring
+NO_STRIP = NO_SPECIAL | binding.DIV_FLAG_NO_PLANE_KERNELS                   # general ring, else two-pass
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -128,7 +130,8 @@ def small_input(n, c, h, w, x_dtype, seed):
 
 
 @pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(map(str, c)))
-@pytest.mark.parametrize("flags", [0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS], ids=["default", "lagged", "planes", "general_ring", "two_pass"])
+@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS],
+                         ids=["default", "lagged", "staged", "planes", "general_ring", "two_pass"])
 def test_small_cases_match_the_checker(case, flags):
     n, c, h, w, block, q, xd, ld = case
     x = small_input(n, c, h, w, xd, seed=n + c + h + w + block + q)
@@ -149,18 +152,25 @@ def test_fused_path_is_taken_where_expected():
     """Guards against silently testing only the general kernels."""
     fused = {case: binding.div_plan_query(binding.make_desc(*case)).fused for case in SMALL}
     lagged = {case: binding.div_plan_query(binding.make_desc(*case), LAGGED).fused for case in SMALL}
+    staged = {case: binding.div_plan_query(binding.make_desc(*case), STAGED).fused for case in SMALL}
     special = {case: binding.div_plan_query(binding.make_desc(*case), NO_SPECIAL).fused for case in SMALL}
     for case in SMALL:
         n, c, h, w, block, q, xd, ld = case
         strip_shape = w % 4 == 0 and min(block, max(h, w)) in (4, 8) and q in (2, 4, 8)
         if strip_shape:
             assert fused[case] == 2 and lagged[case] == 3, case
+            # bulk copies need every sample, plane and band to start on a 16-byte boundary
+            sx = 4 if xd == "f32" else 2
+            b = min(block, max(h, w))
+            aligned = (c * h * w * sx) % 16 == 0 and (h * w * sx) % 16 == 0 and (b * w * sx) % 16 == 0
+            assert staged[case] == (6 if aligned else (4 if planes_shape(case) else 1)), case
         elif planes_shape(case):
-            assert fused[case] == 4 and lagged[case] == 4, case
+            assert fused[case] == 4 and lagged[case] == 4 and staged[case] == 4, case
         else:
-            assert fused[case] in (0, 1) and lagged[case] == fused[case], case
+            assert fused[case] in (0, 1) and lagged[case] == fused[case] and staged[case] == fused[case], case
         assert special[case] == (4 if planes_shape(case) else binding.div_plan_query(binding.make_desc(*case), NO_STRIP).fused), case
     assert sum(1 for c in SMALL if fused[c] == 2) >= 12
+    assert sum(1 for c in SMALL if staged[c] == 6) >= 12
     assert sum(1 for c in SMALL if fused[c] == 4) >= 5
     assert sum(1 for c in SMALL if special[c] == 4) >= 12
     assert fused[(2, 4, 32, 32, 8, 1, "f32", "f32")] == 1          # Q = 1: general ring kernel
@@ -173,9 +183,10 @@ def test_fused_path_is_taken_where_expected():
     for spec in synth.config2() + synth.config1() + synth.config3():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
         big = spec.numel * (4 if spec.x_dtype == "f32" else 2) >= 40 * 2 ** 20
-        assert binding.div_plan_query(d).fused == ((3 if big else 2) if spec.w % 4 == 0 else 4), spec.label()
+        assert binding.div_plan_query(d).fused == ((6 if big else 2) if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
+        assert binding.div_plan_query(d, STAGED).fused == (6 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d).decompress_fast == (1 if spec.w % 4 == 0 else 2)
 
 
@@ -194,7 +205,7 @@ def test_decompress_reads_a_checker_blob():
 def test_degenerate_inputs():
     # constant tensor: residual identically zero, Delta = 0, exact reconstruction
     x = np.full((2, 4, 16, 16), 1.7, dtype=np.float32)
-    for flags in (0, LAGGED, TWO_PASS):
+    for flags in (0, LAGGED, STAGED, TWO_PASS):
         codec, blob, xhat = run_gpu(x, 8, 2, 3, flags=flags)
         lfc, words, stats = split_blob(blob, codec.layout, "f32")
         assert not words.any() and not stats.any()
@@ -227,7 +238,7 @@ def test_same_seed_same_bytes_other_seed_other_codes():
     assert (wa != wc).mean() > 0.5
 
 
-@pytest.mark.parametrize("flags", [0, LAGGED], ids=["strip_ring", "lagged"])
+@pytest.mark.parametrize("flags", [0, LAGGED, STAGED], ids=["strip_ring", "lagged", "staged"])
 def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
     """Failure detection without a fault: the kernel waits for arrivals that never come, its 2 ms limit
     runs out, it records the timeout in the status word and returns; the context stays usable."""
@@ -235,7 +246,7 @@ def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
     spec = synth.config0()[0]
     x = to_device(synth.make_input(spec), "f32")
     codec = binding.Codec(*spec.shape, spec.block, spec.qbits)
-    assert codec.plan(flags).fused == (3 if flags else 2)
+    assert codec.plan(flags).fused == {0: 2, LAGGED: 3, STAGED: 6}[flags]
     st = binding.lib().div_debug_compress_starved(
         ctypes.byref(codec.desc), ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(codec.blob.data_ptr()), codec.blob.numel(),
         ctypes.c_void_p(codec.workspace.data_ptr()), codec.workspace.numel(), 0, ctypes.c_void_p(binding.current_stream_handle()),
@@ -257,7 +268,7 @@ def test_guard_bands_stay_untouched():
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
                  (2, 8, 32, 32, 8, 2, "bf16", "bf16")]:
         n, c, h, w, block, q, xd, ld = case
-        for flags in (0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
+        for flags in (0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
             x = small_input(n, c, h, w, xd, seed=7)
             codec = binding.Codec(n, c, h, w, block, q, xd, ld)
             pad = 4096
@@ -310,7 +321,7 @@ def assert_sampled_parity(spec, seed, sample_ids, flags=0):
 def test_config0_full():
     spec = synth.config0()[0]
     x = synth.make_input(spec)
-    for flags in (0, LAGGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
+    for flags in (0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
         assert_full_parity(x, spec.block, spec.qbits, 0, flags=flags)
 
 
@@ -330,6 +341,7 @@ def test_config2_other_paths_on_one_tensor():
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=NO_STRIP)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=LAGGED)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=RING)
+    assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=STAGED)
     assert_sampled_parity(synth.config2()[0], 0, [17], flags=RING)
 
 
