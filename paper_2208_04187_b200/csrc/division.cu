@@ -267,7 +267,7 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
         out->grid = ch.sp.grid;
         out->threads = ch.sp.threads;
         out->stages = (int32_t)(ch.sp.kr + ch.sp.kq);
-        out->lag = (int32_t)ch.sp.lag_chunks;
+        out->lag = (int32_t)ch.sp.lag_steps;
         out->smem_bytes = ch.sp.smem_bytes;
         out->chunk_elems = ch.sp.chunk_elems;
         out->chunks_per_sample = ch.sp.chunks_per_sample;

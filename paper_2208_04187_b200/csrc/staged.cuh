@@ -8,33 +8,40 @@
 // into two shared-memory rings, issued far ahead by two producer threads, and the worker warps touch
 // shared memory only.
 //
-//   * a CHUNK is a run of G tile row bands of one sample, contiguous in memory (about 28 KB).  Chunks are
-//     claimed from a counter in global scratch.  The CTA that claims chunk j brings chunk j into its
-//     reduce ring (L2 hint: keep) and chunk j - D into its quantise ring (L2 hint: release), D chunks
-//     being at least one sample and about 16 MB of x, which the L2 still holds.
+//   * a CHUNK is a run of G tile row bands of one sample, contiguous in memory (about 28 KB).  Chunk j
+//     belongs to CTA j mod gridDim.x, so the CTAs sweep the tensor together, one round of gridDim.x chunks
+//     after the other.  A CTA brings its i-th chunk into its reduce ring (L2 hint: keep) and, L rounds
+//     later, the same chunk into its quantise ring (L2 hint: release).  L rounds are at least a sample
+//     plus a round, and about 16 MB of x, which the L2 still holds.
 //   * a STRIP is 4 adjacent columns of one band (4 x B elements), owned by one lane: B 16-byte
 //     shared-memory loads, column sums in registers, one shuffle to meet the other half of a B = 8 tile.
 //     Where a strip sits inside a chunk is the same for every chunk, so it comes from a table built once
-//     per CTA.  A UNIT is 32 strips; the units of the chunks are dealt round-robin to the worker warps.
+//     per CTA.  A UNIT is 32 strips.  A CTA's work is the sequence of steps s = 0, 1, ...: the reduce units
+//     of its chunk s, then the quantise units of its chunk s - L; the units are dealt round-robin to the
+//     worker warps, each of which takes its units in order.
 //   * reduce unit: tile mean in the fixed order, stored low-frequency value, extremes of the residual; the
 //     last unit of a chunk folds the chunk's extremes into the sample's slot in global scratch and counts
-//     the chunk as arrived; the arrival that completes a sample derives (delta, Delta, scale), writes the
-//     first two to the blob and publishes delta and scale as one 64-bit word in the slot.
-//   * quantise unit: the tile mean is computed again from the staged rows (cheaper than fetching it from
-//     the other CTA that stored it), then the 4 codes of each strip row are emitted as one byte (Q = 2),
-//     half-word (Q = 4) or word (Q = 8); lanes of a warp write consecutive bytes.  The quantise producer
-//     reads the sample's published word before it issues the copy (bounded wait; normally the first look
-//     succeeds) and posts it beside the stage.
+//     the chunk as arrived (the count is sent by the CTA's watcher thread, behind a release fence).  The
+//     watcher also polls the counts of the samples blockIdx.x, blockIdx.x + gridDim.x, ...; when a sample is
+//     complete it derives (delta, Delta, scale), writes the first two to the blob and publishes delta and
+//     scale as one 64-bit word in the slot.
+//   * quantise unit: the tile mean is computed again from the staged rows, then the 4 codes of each strip
+//     row are emitted as one byte (Q = 2), half-word (Q = 4) or word (Q = 8); lanes of a warp write
+//     consecutive bytes.  The quantise producer reads the sample's published word before it issues the
+//     copy (bounded wait; the look-up is started two chunks ahead, so normally it has long arrived) and
+//     posts it beside the stage.
 //
 // The launch is cooperative so that all CTAs are resident; no grid-wide barrier is used.  Every wait is
 // bounded: when a limit runs out the kernel records DIV_ERR_TIMEOUT in the workspace status word, stops
 // waiting everywhere, lets its own copies land and returns.
 //
-// Why no wait can last: a CTA's workers take units in order, reduce units of a step before its quantise
-// unit, and the quantise producer of a CTA that holds claim j waits for the sample of chunk j - D only.
-// D is at least a sample, so every chunk of that sample has an index below j: it has been claimed, and
-// its claimer is not waiting for it (what a CTA has claimed and not yet reduced lies at or after its own
-// j).  By induction over the samples in order, the sample completes.
+// Why no wait can last: the watchers wait for counts and nobody waits for them but the quantise producers;
+// the only other wait on other CTAs is the quantise producer's, for the sample of its chunk s - L.  The chunks of that sample lie in rounds up to s - L + ceil((S - 1) / gridDim.x) <= s - 1 (S chunks
+// per sample; L is chosen that large).  Take the first sample that is not complete and one of its chunks
+// that has not been reduced, chunk t of CTA Y.  Y's reduce producer issues its copies in order and waits only
+// for its own workers; Y's workers take units in order, and the only thing they can be stuck on is a
+// quantise chunk that Y's quantise producer has not issued, chunk u - L with u <= t.  But that producer waits
+// for a sample whose chunks all lie in rounds before u, i.e. for an earlier sample, which is complete.
 #pragma once
 
 #include "lagged.cuh"
@@ -42,18 +49,28 @@
 namespace divk {
 
 #ifndef DIVK_S_WORKER_WARPS
-#define DIVK_S_WORKER_WARPS 22
+#define DIVK_S_WORKER_WARPS 29
+#endif
+#ifndef DIVK_S_AHEAD
+#define DIVK_S_AHEAD 4
+#endif
+#ifndef DIVK_S_REDUCE_WARPS
+#define DIVK_S_REDUCE_WARPS 14
 #endif
 #ifndef DIVK_S_TARGET_BYTES
 #define DIVK_S_TARGET_BYTES (28 * 1024)
 #endif
 #ifndef DIVK_S_LAG_BYTES
-#define DIVK_S_LAG_BYTES (16u << 20)
+#define DIVK_S_LAG_BYTES (48u << 20)
 #endif
 constexpr int S_WORKER_WARPS = DIVK_S_WORKER_WARPS;
-constexpr int S_THREADS = 32 * (2 + S_WORKER_WARPS);
+constexpr int S_REDUCE_WARPS = DIVK_S_REDUCE_WARPS;      // of the worker warps
+static_assert(S_REDUCE_WARPS >= 1 && S_REDUCE_WARPS < S_WORKER_WARPS, "both worker classes need a warp");
+constexpr int S_SERVICE_WARPS = 3;          // reduce producer, quantise producer, watcher
+constexpr int S_THREADS = 32 * (S_SERVICE_WARPS + S_WORKER_WARPS);
 constexpr int S_MAX_STAGES = 8;
-constexpr uint32_t S_CLAIM_RING = 32;
+constexpr uint32_t S_MAILBOX = 16;
+constexpr int S_AHEAD = DIVK_S_AHEAD;       // chunks the reduce half may lead the quantise half by, beyond the lag
 
 struct SPlan {
     int32_t grid, threads, smem_bytes;
@@ -66,7 +83,7 @@ struct SPlan {
     uint32_t chunks_per_sample;    // S
     uint32_t bands_per_sample;     // C * Hb
     uint32_t stage_bytes;
-    uint32_t lag_chunks;           // D
+    uint32_t lag_steps;            // L: rounds between the reduce and the quantise half of a chunk
     uint32_t uniform;              // 1: every band has B rows (H % B == 0); 0: chunks are whole planes
     uint64_t total_chunks;
 };
@@ -91,10 +108,10 @@ struct SParams {
 
 // what a producer posts beside a stage before it issues the copy
 struct SDesc {
-    uint32_t nslots;               // strip slots of the chunk (0: the step has no chunk for this ring)
+    uint32_t nslots;               // strip slots of the chunk
     uint32_t n;                    // sample
     uint32_t tile0;                // first tile of the chunk inside the sample
-    uint32_t seq;                  // 1 + the step whose chunk the stage holds; written last (see s_wait_step)
+    uint32_t seq;                  // 1 + index (in this CTA's list) of the chunk the stage holds; written last (see s_wait_chunk)
     uint64_t quad0;                // (n * CHW + e0) / 4: first group of 4 elements of the chunk in the tensor
     uint64_t ctr0;                 // counter of the random stream of that group, minus K_GROUP (see rng_group)
     float delta, scale;            // quantise ring only
@@ -106,13 +123,16 @@ struct SCtl {
     SDesc desc_r[S_MAX_STAGES], desc_q[S_MAX_STAGES];
     uint32_t kmin[S_MAX_STAGES], kmax[S_MAX_STAGES];      // ~key(min r), key(max r) folded over the units of a chunk
     uint32_t done_r[S_MAX_STAGES], done_q[S_MAX_STAGES];  // units of the chunk that are finished
-    uint32_t claims[S_CLAIM_RING];                        // claimed chunk index of step i at [i % S_CLAIM_RING]
-    uint32_t claims_n;                                    // steps published by the reduce producer
-    uint32_t q_steps;                                     // steps taken over by the quantise producer
-    uint32_t end_step;                                    // first step that does not exist (0xFFFFFFFF: not known yet)
+    uint32_t q_closed;                                    // chunks whose quantise half is finished
+    uint32_t mb_n[S_MAILBOX], mb_seq[S_MAILBOX];          // reduce closers -> watcher: chunk it of this CTA (slot it % S_MAILBOX)
+                                                          // has been folded into sample mb_n; mb_seq = it + 1, written last
+    uint32_t mb_done;                                     // chunks the watcher has counted
     uint32_t failed;
 };
 
+__device__ __forceinline__ void red_add_relaxed(uint32_t* p, uint32_t v) {
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar,
                                                uint64_t policy) {
     asm volatile(
@@ -122,11 +142,27 @@ __device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gmem_
         : "memory");
 }
 
-__device__ __forceinline__ bool s_give_up(const SParams& p, SCtl* ctl, uint64_t& t0) {
+// Bounded waits.  The polling loops below stay on chip: a look at the clock every few polls, and only once a
+// wait has lasted S_SLOW_CYCLES (far longer than any wait of a healthy run) the slow check, which reads the
+// status word in global memory (has any wait of this launch given up?) and the wall clock.
+constexpr long long S_SLOW_CYCLES = 1ll << 15;
+struct SWait {
+    long long c0;        // clock at the last slow check (0: none yet)
+    uint64_t t0;         // wall clock at the first slow check
+};
+__device__ __forceinline__ bool s_give_up(const SParams& p, SCtl* ctl, SWait& w) {
+    const long long c = clock64();
+    if (w.c0 == 0) {
+        w.c0 = c;
+        w.t0 = 0;
+        return false;
+    }
+    if (c - w.c0 < S_SLOW_CYCLES) return false;
+    w.c0 = c;
     if (lds_volatile(&ctl->failed) || ld_relaxed_u32(p.ws) != 0u) return true;
     const uint64_t t = now_ns();
-    if (t0 == 0) t0 = t;
-    return t - t0 > p.timeout_ns;
+    if (w.t0 == 0) w.t0 = t;
+    return t - w.t0 > p.timeout_ns;
 }
 __device__ __forceinline__ void s_record_failure(const SParams& p, SCtl* ctl, uint32_t detail) {
     atomicCAS(p.ws, 0u, (uint32_t)DIV_ERR_TIMEOUT);
@@ -137,35 +173,35 @@ __device__ __forceinline__ void s_record_failure(const SParams& p, SCtl* ctl, ui
 __device__ __forceinline__ bool s_wait(uint64_t* bar, uint32_t parity, const SParams& p, SCtl* ctl, uint32_t detail) {
     if (mbar_try_wait(bar, parity)) return true;
     uint32_t polls = 0;
-    uint64_t t0 = 0;
+    SWait w = {0, 0};
     while (!mbar_try_wait(bar, parity)) {
-        if ((++polls & 31u) == 0 && s_give_up(p, ctl, t0)) {
+        if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
             s_record_failure(p, ctl, detail);
             return false;
         }
     }
     return true;
 }
-// worker side: wait for the chunk of `step`; false when the step does not exist or a wait gave up.
-// Worker warps skip steps (units are dealt round-robin), so a warp may look at a stage a whole turn of the
+// worker side: wait for the CTA's chunk number `it` in a ring; false when a wait gave up.
+// Worker warps skip chunks (units are dealt round-robin), so a warp may look at a stage a whole turn of the
 // ring before the producer does, when the barrier's phase of that parity is still the one two turns back,
 // which counts as complete.  Hence the sequence number: the parity wait starts only once the producer has
-// posted this step's descriptor and its arrival on the barrier.
-__device__ __forceinline__ bool s_wait_step(uint64_t* bar, uint32_t parity, const uint32_t* seq, uint32_t step,
-                                            const SParams& p, SCtl* ctl) {
+// posted this chunk's descriptor and its arrival on the barrier.
+__device__ __forceinline__ bool s_wait_chunk(uint64_t* bar, uint32_t parity, const uint32_t* seq, uint32_t it,
+                                             const SParams& p, SCtl* ctl) {
     uint32_t polls = 0;
-    uint64_t t0 = 0;
-    while (lds_volatile(seq) != step + 1u) {
-        if (lds_volatile(&ctl->end_step) <= step) return false;
-        if ((++polls & 63u) == 0 && s_give_up(p, ctl, t0)) {
-            s_record_failure(p, ctl, 0x40000000u | step);
+    SWait w = {0, 0};
+    while (lds_volatile(seq) != it + 1u) {
+        __nanosleep(32);
+        if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+            s_record_failure(p, ctl, 0x40000000u | it);
             return false;
         }
     }
     __threadfence_block();
     while (!mbar_try_wait(bar, parity)) {
-        if ((++polls & 63u) == 0 && s_give_up(p, ctl, t0)) {
-            s_record_failure(p, ctl, 0x40000000u | step);
+        if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+            s_record_failure(p, ctl, 0x40000000u | it);
             return false;
         }
     }
@@ -235,17 +271,20 @@ staged_kernel(const SParams p) {
     const uint32_t stage_bytes = p.pl.stage_bytes;
     unsigned char* ring_r = smem;
     unsigned char* ring_q = smem + (size_t)KR * stage_bytes;
-    uint2* table = reinterpret_cast<uint2*>(ring_q + (size_t)KQ * stage_bytes);
-    SCtl* ctl = reinterpret_cast<SCtl*>(reinterpret_cast<unsigned char*>(table) + (((size_t)p.pl.slots * 8u + 15u) & ~(size_t)15u));
+    uint32_t* table = reinterpret_cast<uint32_t*>(ring_q + (size_t)KQ * stage_bytes);
+    SCtl* ctl = reinterpret_cast<SCtl*>(reinterpret_cast<unsigned char*>(table) + (((size_t)p.pl.slots * 4u + 15u) & ~(size_t)15u));
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t S = p.pl.chunks_per_sample;
     const uint32_t TU = (uint32_t)p.pl.total_chunks;      // < 2^30 (checked by the planner)
-    const uint32_t D = p.pl.lag_chunks;
+    const uint32_t L = p.pl.lag_steps;
+    const uint32_t G = gridDim.x;
+    // this CTA's chunks: blockIdx.x + it * G for it < n_my
+    const uint32_t n_my = blockIdx.x < TU ? (TU - blockIdx.x + G - 1u) / G : 0u;
 
     // ---- set-up: strip table, barriers ----
-    //   x: offset of the strip's first element inside the chunk, in groups of 4 elements
-    //   y: in-bounds rows (0: padding slot) | kind of tile << 4 | writes the tile's mean << 6 | tile inside the chunk << 8
+    //   bits 0-12 offset of the strip's first element inside the chunk, in groups of 4 elements; 13-16 in-bounds rows
+    //   (0: padding slot); 17-18 kind of tile; 19 writes the tile's mean; 20-31 tile inside the chunk
     for (uint32_t sl = threadIdx.x; sl < p.pl.slots; sl += blockDim.x) {
         const uint32_t band = sl / p.pl.spb, q = sl - band * p.pl.spb;
         const uint32_t col0 = 4u * q;
@@ -262,7 +301,7 @@ staged_kernel(const SParams p) {
         const uint32_t bw = q / LPT;
         const uint32_t which = ((rows != s.B) ? 2u : 0u) + ((bw == s.Wb - 1u && (s.W % s.B) != 0u) ? 1u : 0u);
         const uint32_t writer = (q % LPT) == 0 ? 1u : 0u;
-        table[sl] = make_uint2(ok ? (eoff >> 2) : 0u, (ok ? rows : 0u) | (which << 4) | (writer << 6) | ((band * s.Wb + bw) << 8));
+        table[sl] = (ok ? (eoff >> 2) : 0u) | ((ok ? rows : 0u) << 13) | (which << 17) | (writer << 19) | ((band * s.Wb + bw) << 20);
     }
     if (threadIdx.x == 0) {
         for (uint32_t i = 0; i < (uint32_t)S_MAX_STAGES; ++i) {
@@ -277,371 +316,341 @@ staged_kernel(const SParams p) {
             ctl->desc_r[i].seq = 0;
             ctl->desc_q[i].seq = 0;
         }
-        ctl->claims_n = 0;
-        ctl->q_steps = 0;
-        ctl->end_step = 0xFFFFFFFFu;
+        ctl->q_closed = 0;
+        ctl->mb_done = 0;
+        for (uint32_t i = 0; i < S_MAILBOX; ++i) ctl->mb_seq[i] = 0;
         ctl->failed = 0;
         fence_barrier_init();
     }
     __syncthreads();
 
-    if (warp == 0) {
-        // ================= reduce producer: claims chunks, streams them from HBM =================
-        if (lane == 0) {
-            uint32_t* claim_word = p.ws + WS_CLAIM_WORD;
-            const uint64_t pol_keep = l2_policy_keep();
-            uint32_t i = 0;
-            uint32_t j = atomicAdd(claim_word, 1u);
-            bool ok = true;
-            while (j < TU + D) {
-                const uint32_t jn = atomicAdd(claim_word, 1u);          // needed only at the next turn
-                // hand the claim to the quantise producer
-                {
-                    uint32_t polls = 0;
-                    uint64_t t0 = 0;
-                    while (i - lds_volatile(&ctl->q_steps) >= S_CLAIM_RING) {
-                        if ((++polls & 31u) == 0 && s_give_up(p, ctl, t0)) {
-                            s_record_failure(p, ctl, 0x80000001u);
-                            ok = false;
-                            break;
-                        }
-                    }
-                    if (!ok) break;
-                }
-                ctl->claims[i % S_CLAIM_RING] = j;
+    if (warp == 2) {
+        // ================= watcher (one thread).  Two duties, taken in turns:
+        //   * count this CTA's folded chunks as arrived: the reduce closers post them in a mailbox; the watcher
+        //     takes what is there, issues ONE release fence at gpu scope (the closers' folds happen before their
+        //     posts, so the fence orders them before the counts; it costs a round trip to the L2, which is why
+        //     no reduce warp issues it) and sends the counts, reductions without an answer;
+        //   * complete the samples n = blockIdx.x, blockIdx.x + gridDim.x, ...: when every chunk of the sample has
+        //     been counted, derive (delta, Delta, scale) from the folded extremes, write the first two to the blob
+        //     and publish delta and scale in the slot.
+        if (lane != 0) return;
+        uint32_t next = 0;                       // next chunk of this CTA to count
+        uint32_t n = blockIdx.x;                 // next sample to complete
+        uint32_t polls = 0;
+        SWait w = {0, 0};
+        while (next < n_my || n < s.N) {
+            bool progress = false;
+            uint32_t cnt = 0;
+            while (next + cnt < n_my && cnt < S_MAILBOX && lds_volatile(&ctl->mb_seq[(next + cnt) % S_MAILBOX]) == next + cnt + 1u) ++cnt;
+            if (cnt) {
                 __threadfence_block();
-                sts_volatile(&ctl->claims_n, i + 1u);
-                const uint32_t round = fdiv(i, p.by_kr);
-                const uint32_t st = i - round * KR;
-                if (i >= KR && !s_wait(&ctl->empty_r[st], (round - 1u) & 1u, p, ctl, 0x80000002u)) {
-                    ok = false;
-                    break;
-                }
-                SDesc d;
-                d.nslots = 0;
-                d.n = 0;
-                d.tile0 = 0;
-                d.seq = 0;
-                d.quad0 = 0;
-                d.ctr0 = 0;
-                d.delta = 0.f;
-                d.scale = 0.f;
-                if (j < TU) {
-                    const uint32_t n = fdiv(j, p.by_S);
-                    const uint32_t k = j - n * S;
-                    const uint32_t e0 = k * p.pl.chunk_elems;
-                    const uint32_t nelem = min(p.pl.chunk_elems, s.CHW - e0);
-                    const uint32_t nbands = min(p.pl.G, p.pl.bands_per_sample - k * p.pl.G);
-                    d.nslots = nbands * p.pl.spb;
-                    d.n = n;
-                    d.tile0 = k * p.pl.G * s.Wb;
-                    ctl->desc_r[st] = d;
-                    const uint32_t bytes = nelem * (uint32_t)sizeof(XT);
-                    const XT* src = reinterpret_cast<const XT*>(p.x) + ((size_t)n * s.CHW + e0);
-                    mbar_arrive_expect_tx(&ctl->full_r[st], bytes);
-                    bulk_load_hint(ring_r + (size_t)st * stage_bytes, src, bytes, &ctl->full_r[st], pol_keep);
-                } else {
-                    ctl->desc_r[st] = d;
-                    mbar_arrive(&ctl->full_r[st]);
-                }
+                fence_acq_rel_gpu();
+                for (uint32_t i = 0; i < cnt; ++i)
+                    red_add_relaxed(p.ws + WS_HEADER_WORDS + (size_t)ctl->mb_n[(next + i) % S_MAILBOX] * WS_SLOT_WORDS + 2, 1u);
+                next += cnt;
                 __threadfence_block();
-                sts_volatile(&ctl->desc_r[st].seq, i + 1u);
-                ++i;
-                j = jn;
+                sts_volatile(&ctl->mb_done, next);
+                progress = true;
             }
+            if (n < s.N) {
+                uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+                if (ld_acquire_u32(slot + 2) == p.expected_chunks) {
+                    const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
+                    p.stats[2 * (size_t)n + 0] = qp.delta;
+                    p.stats[2 * (size_t)n + 1] = qp.step;
+                    const uint64_t word = ((uint64_t)(__float_as_uint(qp.scale) | 0x80000000u) << 32) | (uint64_t)__float_as_uint(qp.delta);
+                    st_release_u64(reinterpret_cast<uint64_t*>(slot + 4), word);
+                    n += G;
+                    progress = true;
+                }
+            } else if (!cnt) {
+                __nanosleep(100);
+            }
+            if (progress) {
+                polls = 0;
+                w.c0 = 0;
+            } else if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+                s_record_failure(p, ctl, n < s.N ? n + 1u : 0x80000007u);
+                break;
+            }
+        }
+        return;
+    }
+
+    if (warp < 2) {
+        // ================= producers: warp 0 streams the chunks from HBM into the reduce ring, warp 1 streams
+        // ================= them again, from L2 and with their sample's parameters, into the quantise ring
+        if (lane != 0) return;
+        const bool quant = warp == 1;
+        const uint32_t K = quant ? KQ : KR;
+        const FastDiv by_K = quant ? p.by_kq : p.by_kr;
+        uint64_t* full = quant ? ctl->full_q : ctl->full_r;
+        uint64_t* empty = quant ? ctl->empty_q : ctl->empty_r;
+        SDesc* desc = quant ? ctl->desc_q : ctl->desc_r;
+        unsigned char* ring = quant ? ring_q : ring_r;
+        const uint64_t policy = quant ? l2_policy_release() : l2_policy_keep();
+        // parameter words of the samples of the next two chunks, asked for ahead of time
+        uint64_t w0 = 0, w1 = 0;
+        if (quant) {
+            if (n_my > 0u) w0 = ld_relaxed_u64(reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)fdiv(blockIdx.x, p.by_S) * WS_SLOT_WORDS + 4));
+            if (n_my > 1u) w1 = ld_relaxed_u64(reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)fdiv(blockIdx.x + G, p.by_S) * WS_SLOT_WORDS + 4));
+        }
+        uint32_t it = 0;
+        bool ok = true;
+        for (; it < n_my; ++it) {
+            const uint32_t round = fdiv(it, by_K);
+            const uint32_t st = it - round * K;
+            const uint32_t j = blockIdx.x + it * G;
+            const uint32_t n = fdiv(j, p.by_S);
+            const uint32_t k = j - n * S;
+            uint64_t word = w0;
+            if (quant) {
+                w0 = w1;
+                if (it + 2u < n_my)
+                    w1 = ld_relaxed_u64(reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)fdiv(j + 2u * G, p.by_S) * WS_SLOT_WORDS + 4));
+            }
+            if (it >= K && !s_wait(&empty[st], (round - 1u) & 1u, p, ctl, 0x80000002u + (quant ? 2u : 0u))) {
+                ok = false;
+                break;
+            }
+            if (!quant && it >= L + (uint32_t)S_AHEAD) {
+                // the first read must not run away from the second one: what it brought into the L2 would be gone
+                // by the time it is read again.  (The quantise half of chunk c needs reduce halves up to round
+                // c + L - 1 only, so this wait always ends.)
+                uint32_t polls = 0;
+                SWait w = {0, 0};
+                while (it - lds_volatile(&ctl->q_closed) >= L + (uint32_t)S_AHEAD) {
+                    __nanosleep(32);
+                    if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+                        s_record_failure(p, ctl, 0x80000006u);
+                        ok = false;
+                        break;
+                    }
+                }
+                if (!ok) break;
+            }
+            if (quant && !(word >> 63)) {
+                const uint64_t* pw = reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS + 4);
+                uint32_t polls = 0;
+                SWait w = {0, 0};
+                while (true) {
+                    word = ld_relaxed_u64(pw);
+                    if (word >> 63) break;
+                    if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+                        s_record_failure(p, ctl, n + 1u);
+                        ok = false;
+                        break;
+                    }
+                    __nanosleep(100);
+                }
+                if (!ok) break;
+            }
+            const uint32_t e0 = k * p.pl.chunk_elems;
+            const uint32_t nelem = min(p.pl.chunk_elems, s.CHW - e0);
+            const uint32_t nbands = min(p.pl.G, p.pl.bands_per_sample - k * p.pl.G);
+            SDesc d;
+            d.nslots = nbands * p.pl.spb;
+            d.n = n;
+            d.tile0 = k * p.pl.G * s.Wb;
+            d.seq = 0;
+            d.quad0 = ((uint64_t)n * s.CHW + e0) >> 2;
+            d.ctr0 = rng_sample_base(p.seed, n) + K_GROUP * (uint64_t)((e0 >> 2) + 1u);
+            d.delta = __uint_as_float((uint32_t)word);
+            d.scale = __uint_as_float((uint32_t)(word >> 32) & 0x7FFFFFFFu);
+            desc[st] = d;
+            const uint32_t bytes = nelem * (uint32_t)sizeof(XT);
+            const XT* src = reinterpret_cast<const XT*>(p.x) + ((size_t)n * s.CHW + e0);
+            mbar_arrive_expect_tx(&full[st], bytes);
+            bulk_load_hint(ring + (size_t)st * stage_bytes, src, bytes, &full[st], policy);
             __threadfence_block();
-            sts_volatile(&ctl->end_step, i);
-            if (!ok || lds_volatile(&ctl->failed)) {
-                // a wait gave up somewhere: let the copies still in flight land before the CTA may exit
-                const uint32_t first = i > KR ? i - KR : 0u;
-                for (uint32_t t = first; t < i; ++t) {
-                    const uint32_t round = fdiv(t, p.by_kr);
-                    uint32_t polls = 0;
-                    while (!mbar_try_wait(&ctl->full_r[t - round * KR], round & 1u) && ++polls < (1u << 20)) {
-                    }
+            sts_volatile(&desc[st].seq, it + 1u);
+        }
+        if (!ok || lds_volatile(&ctl->failed)) {
+            // a wait gave up somewhere: let the copies still in flight land before the CTA may exit
+            const uint32_t first = it > K ? it - K : 0u;
+            for (uint32_t t = first; t < it; ++t) {
+                const uint32_t round = fdiv(t, by_K);
+                uint32_t polls = 0;
+                while (!mbar_try_wait(&full[t - round * K], round & 1u) && ++polls < (1u << 20)) {
                 }
             }
         }
         return;
     }
 
-    if (warp == 1) {
-        // ================= quantise producer: chunk j - D from L2, with its sample's parameters =================
-        if (lane == 0) {
-            const uint64_t pol_release = l2_policy_release();
-            uint32_t i = 0;
-            bool ok = true;
-            uint64_t pre_word = 0;          // parameter word looked up ahead of time for step pre_step
-            uint32_t pre_step = 0xFFFFFFFFu;
-            while (true) {
-                // the claim of step i
-                {
-                    uint32_t polls = 0;
-                    uint64_t t0 = 0;
-                    bool ended = false;
-                    while (lds_volatile(&ctl->claims_n) <= i) {
-                        if (lds_volatile(&ctl->end_step) <= i) {
-                            ended = true;
-                            break;
-                        }
-                        if ((++polls & 31u) == 0 && s_give_up(p, ctl, t0)) {
-                            s_record_failure(p, ctl, 0x80000003u);
-                            ok = false;
-                            break;
-                        }
-                    }
-                    if (ended || !ok) break;
-                }
-                __threadfence_block();
-                const uint32_t j = ctl->claims[i % S_CLAIM_RING];
-                // look ahead: the claim of the next step, if it is there already
-                uint32_t jnext = 0xFFFFFFFFu;
-                if (lds_volatile(&ctl->claims_n) > i + 1u) jnext = ctl->claims[(i + 1u) % S_CLAIM_RING];
-                __threadfence_block();
-                sts_volatile(&ctl->q_steps, i + 1u);
-
-                const bool has = j >= D && j - D < TU;
-                uint32_t n = 0, k = 0;
-                uint64_t word = 0;
-                if (has) {
-                    n = fdiv(j - D, p.by_S);
-                    k = (j - D) - n * S;
-                    const uint64_t* pw = reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS + 4);
-                    word = (pre_step == i) ? pre_word : ld_relaxed_u64(pw);
-                }
-                // issue the look-up for the next step now; its answer is used a turn later
-                if (jnext != 0xFFFFFFFFu && jnext >= D && jnext - D < TU) {
-                    const uint32_t nn = fdiv(jnext - D, p.by_S);
-                    pre_word = ld_relaxed_u64(reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)nn * WS_SLOT_WORDS + 4));
-                    pre_step = i + 1u;
-                }
-                const uint32_t round = fdiv(i, p.by_kq);
-                const uint32_t st = i - round * KQ;
-                if (i >= KQ && !s_wait(&ctl->empty_q[st], (round - 1u) & 1u, p, ctl, 0x80000004u)) {
-                    ok = false;
-                    break;
-                }
-                SDesc d;
-                d.nslots = 0;
-                d.n = 0;
-                d.tile0 = 0;
-                d.seq = 0;
-                d.quad0 = 0;
-                d.ctr0 = 0;
-                d.delta = 0.f;
-                d.scale = 0.f;
-                if (has) {
-                    if (!(word >> 63)) {
-                        const uint64_t* pw = reinterpret_cast<const uint64_t*>(p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS + 4);
-                        uint32_t polls = 0;
-                        uint64_t t0 = 0;
-                        while (true) {
-                            word = ld_relaxed_u64(pw);
-                            if (word >> 63) break;
-                            if ((++polls & 7u) == 0 && s_give_up(p, ctl, t0)) {
-                                s_record_failure(p, ctl, n + 1u);
-                                ok = false;
-                                break;
-                            }
-                            __nanosleep(100);
-                        }
-                        if (!ok) break;
-                    }
-                    const uint32_t e0 = k * p.pl.chunk_elems;
-                    const uint32_t nelem = min(p.pl.chunk_elems, s.CHW - e0);
-                    const uint32_t nbands = min(p.pl.G, p.pl.bands_per_sample - k * p.pl.G);
-                    d.nslots = nbands * p.pl.spb;
-                    d.n = n;
-                    d.tile0 = k * p.pl.G * s.Wb;
-                    d.quad0 = ((uint64_t)n * s.CHW + e0) >> 2;
-                    d.ctr0 = rng_sample_base(p.seed, n) + K_GROUP * (uint64_t)((e0 >> 2) + 1u);
-                    d.delta = __uint_as_float((uint32_t)word);
-                    d.scale = __uint_as_float((uint32_t)(word >> 32) & 0x7FFFFFFFu);
-                    ctl->desc_q[st] = d;
-                    const uint32_t bytes = nelem * (uint32_t)sizeof(XT);
-                    const XT* src = reinterpret_cast<const XT*>(p.x) + ((size_t)n * s.CHW + e0);
-                    mbar_arrive_expect_tx(&ctl->full_q[st], bytes);
-                    bulk_load_hint(ring_q + (size_t)st * stage_bytes, src, bytes, &ctl->full_q[st], pol_release);
-                } else {
-                    ctl->desc_q[st] = d;
-                    mbar_arrive(&ctl->full_q[st]);
-                }
-                __threadfence_block();
-                sts_volatile(&ctl->desc_q[st].seq, i + 1u);
-                ++i;
-            }
-            if (!ok || lds_volatile(&ctl->failed)) {
-                const uint32_t first = i > KQ ? i - KQ : 0u;
-                for (uint32_t t = first; t < i; ++t) {
-                    const uint32_t round = fdiv(t, p.by_kq);
-                    uint32_t polls = 0;
-                    while (!mbar_try_wait(&ctl->full_q[t - round * KQ], round & 1u) && ++polls < (1u << 20)) {
-                    }
-                }
-            }
-        }
-        return;
-    }
-
-    // ================= workers =================
-    const uint32_t NW = (blockDim.x >> 5) - 2;
+    // ================= workers: the first S_REDUCE_WARPS warps take the reduce units, the others the quantise
+    // ================= units, each class dealing its units round-robin and taking them in order
     const uint32_t nf = p.pl.nf;
     const uint32_t row_bytes = s.W * (uint32_t)sizeof(XT);
     const uint32_t W4 = s.W >> 2;
     LT* lfc_out = reinterpret_cast<LT*>(p.lfc);
     OutT* packed = reinterpret_cast<OutT*>(p.packed);
-
-    // unit k of step `step`: k < nf reduce unit k, else quantise unit k - nf
-    uint32_t step = 0, k = warp - 2;
-    while (k >= 2u * nf) {
-        k -= 2u * nf;
-        ++step;
+    const bool reducer = warp < (uint32_t)S_SERVICE_WARPS + (uint32_t)S_REDUCE_WARPS;
+    const uint32_t NW = reducer ? (uint32_t)S_REDUCE_WARPS : (blockDim.x >> 5) - (uint32_t)S_SERVICE_WARPS - (uint32_t)S_REDUCE_WARPS;
+    // unit k of this CTA's chunk number `it`
+    uint32_t it = 0, k = reducer ? warp - (uint32_t)S_SERVICE_WARPS : warp - (uint32_t)S_SERVICE_WARPS - (uint32_t)S_REDUCE_WARPS;
+    while (k >= nf) {
+        k -= nf;
+        ++it;
     }
 
-    while (true) {
-        if (k < nf) {
-            // ---------------- reduce unit ----------------
-            const uint32_t round = fdiv(step, p.by_kr);
-            const uint32_t st = step - round * KR;
-            if (!s_wait_step(&ctl->full_r[st], round & 1u, &ctl->desc_r[st].seq, step, p, ctl)) break;
-            // every unit index of the step takes part in the closing count, also where a short chunk has no
-            // strips for it: a stage is recycled only after each of its nf readers has looked at it
+    if (reducer) {
+        for (; it < n_my;) {
+            const uint32_t round = fdiv(it, p.by_kr);
+            const uint32_t st = it - round * KR;
+            const bool landed = __all_sync(0xFFFFFFFFu, s_wait_chunk(&ctl->full_r[st], round & 1u, &ctl->desc_r[st].seq, it, p, ctl));
+            if (!landed) break;
+            // every unit index takes part in the closing count, also where a short chunk has no strips for it:
+            // a stage is recycled only after each of its nf readers has looked at it
             const uint32_t nslots = ctl->desc_r[st].nslots;
             const bool work = k * 32u < nslots;
-            {
-                uint32_t kmin = 0, kmax = 0;
-                if (work) {
-                    const uint32_t n = ctl->desc_r[st].n;
-                    const uint32_t sl = k * 32u + lane;
-                    uint2 rec = make_uint2(0u, 0u);
-                    if (sl < nslots) rec = table[sl];
-                    const uint32_t rows = rec.y & 15u;
-                    const bool active = rows != 0u;
-                    const uint32_t which = (rec.y >> 4) & 3u;
-                    const unsigned char* xs = ring_r + (size_t)st * stage_bytes + ((size_t)rec.x << QSHIFT);
-                    const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
-                    uint64_t vxy[P2], vzw[P2];
-                    s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
-                    const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
-                    const float stored = Elem<LT>::round(mean);
-                    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-                    if (active) {
-                        if (rec.y & 64u)
-                            Elem<LT>::store(lfc_out + (size_t)n * s.C * s.TPP + ctl->desc_r[st].tile0 + (rec.y >> 8), mean);
-                        // extremes of x over the strip's in-bounds rows; x -> fl(x - stored) is monotone
-                        float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+            uint32_t kmin = 0, kmax = 0;
+            if (work) {
+                const uint32_t n = ctl->desc_r[st].n;
+                const uint32_t sl = k * 32u + lane;
+                uint32_t rec = 0u;
+                if (sl < nslots) rec = table[sl];
+                const uint32_t rows = (rec >> 13) & 15u;
+                const bool active = rows != 0u;
+                const uint32_t which = (rec >> 17) & 3u;
+                const unsigned char* xs = ring_r + (size_t)st * stage_bytes + ((size_t)(rec & 0x1FFFu) << QSHIFT);
+                const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
+                uint64_t vxy[P2], vzw[P2];
+                s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
+                const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
+                const float stored = Elem<LT>::round(mean);
+                float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+                if (active) {
+                    if (rec & (1u << 19))
+                        Elem<LT>::store(lfc_out + (size_t)n * s.C * s.TPP + ctl->desc_r[st].tile0 + (rec >> 20), mean);
+                    // extremes of x over the strip's in-bounds rows; x -> fl(x - stored) is monotone
+                    float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
 #pragma unroll
-                        for (int r = 0; r < P2; ++r) {
-                            if (full || (uint32_t)r < rows) {
-                                float a_, b_, c_, d_;
-                                upk2(vxy[r], a_, b_);
-                                upk2(vzw[r], c_, d_);
-                                blo = fmin3(blo, a_, b_);
-                                blo = fmin3(blo, c_, d_);
-                                bhi = fmax3(bhi, a_, b_);
-                                bhi = fmax3(bhi, c_, d_);
-                            }
+                    for (int r = 0; r < P2; ++r) {
+                        if (full || (uint32_t)r < rows) {
+                            float a_, b_, c_, d_;
+                            upk2(vxy[r], a_, b_);
+                            upk2(vzw[r], c_, d_);
+                            blo = fmin3(blo, a_, b_);
+                            blo = fmin3(blo, c_, d_);
+                            bhi = fmax3(bhi, a_, b_);
+                            bhi = fmax3(bhi, c_, d_);
                         }
-                        lo = __fsub_rn(blo, stored);
-                        hi = __fsub_rn(bhi, stored);
                     }
-                    kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
-                    kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+                    lo = __fsub_rn(blo, stored);
+                    hi = __fsub_rn(bhi, stored);
                 }
-                __syncwarp();
-                if (lane == 0) {
-                    if (work) {
-                        atomicMax(&ctl->kmin[st], kmin);
-                        atomicMax(&ctl->kmax[st], kmax);
-                        __threadfence_block();
-                    }
-                    if (atomicAdd(&ctl->done_r[st], 1u) == nf - 1u) {
-                        // last unit of this chunk: fold the chunk into its sample's slot, hand the stage back
-                        __threadfence_block();
-                        const uint32_t smin = atomicExch(&ctl->kmin[st], 0u);
-                        const uint32_t smax = atomicExch(&ctl->kmax[st], 0u);
-                        ctl->done_r[st] = 0u;
-                        if (nslots && lds_volatile(&ctl->failed) == 0u) {
-                            const uint32_t n = ctl->desc_r[st].n;
-                            uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
-                            red_max_relaxed(slot + 0, smin);
-                            red_max_relaxed(slot + 1, smax);
-                            const uint32_t before = atom_add_acq_rel(slot + 2, 1u);
-                            if (before + 1u == p.expected_chunks) {
-                                // this arrival completes the sample
-                                const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
-                                p.stats[2 * (size_t)n + 0] = qp.delta;
-                                p.stats[2 * (size_t)n + 1] = qp.step;
-                                const uint64_t word = ((uint64_t)(__float_as_uint(qp.scale) | 0x80000000u) << 32) |
-                                                      (uint64_t)__float_as_uint(qp.delta);
-                                st_release_u64(reinterpret_cast<uint64_t*>(slot + 4), word);
+                kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
+                kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (work) {
+                    atomicMax(&ctl->kmin[st], kmin);
+                    atomicMax(&ctl->kmax[st], kmax);
+                    __threadfence_block();
+                }
+                if (atomicAdd(&ctl->done_r[st], 1u) == nf - 1u) {
+                    // last unit of this chunk: fold the chunk into its sample's slot, hand the stage back
+                    __threadfence_block();
+                    const uint32_t smin = atomicExch(&ctl->kmin[st], 0u);
+                    const uint32_t smax = atomicExch(&ctl->kmax[st], 0u);
+                    ctl->done_r[st] = 0u;
+                    const uint32_t n = ctl->desc_r[st].n;
+                    __threadfence_block();
+                    mbar_arrive(&ctl->empty_r[st]);
+                    if (lds_volatile(&ctl->failed) == 0u) {
+                        // fold the chunk's extremes into the sample's slot in global scratch (reductions without an
+                        // answer: an atomic that returns the old count to 148 CTAs was measured to cost more than the
+                        // rest of the kernel) and tell the watcher, who counts the chunk as arrived
+                        uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+                        red_max_relaxed(slot + 0, smin);
+                        red_max_relaxed(slot + 1, smax);
+                        uint32_t polls = 0;
+                        SWait w = {0, 0};
+                        bool room = true;
+                        while (it - lds_volatile(&ctl->mb_done) >= S_MAILBOX) {          // never in practice
+                            __nanosleep(64);
+                            if ((++polls & 7u) == 0 && s_give_up(p, ctl, w)) {
+                                s_record_failure(p, ctl, 0x80000008u);
+                                room = false;
+                                break;
                             }
                         }
-                        __threadfence_block();
-                        mbar_arrive(&ctl->empty_r[st]);
+                        if (room) {
+                            ctl->mb_n[it % S_MAILBOX] = n;
+                            __threadfence_block();
+                            sts_volatile(&ctl->mb_seq[it % S_MAILBOX], it + 1u);
+                        }
                     }
                 }
             }
-        } else {
-            // ---------------- quantise unit ----------------
-            const uint32_t kk = k - nf;
-            const uint32_t round = fdiv(step, p.by_kq);
-            const uint32_t st = step - round * KQ;
-            if (!s_wait_step(&ctl->full_q[st], round & 1u, &ctl->desc_q[st].seq, step, p, ctl)) break;
-            const uint32_t nslots = ctl->desc_q[st].nslots;
-            {
-                if (kk * 32u < nslots) {
-                    const uint32_t sl = kk * 32u + lane;
-                    uint2 rec = make_uint2(0u, 0u);
-                    if (sl < nslots) rec = table[sl];
-                    const uint32_t rows = rec.y & 15u;
-                    const bool active = rows != 0u;
-                    const uint32_t which = (rec.y >> 4) & 3u;
-                    const unsigned char* xs = ring_q + (size_t)st * stage_bytes + ((size_t)rec.x << QSHIFT);
-                    const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
-                    uint64_t vxy[P2], vzw[P2];
-                    s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
-                    const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
-                    const float stored = Elem<LT>::round(mean);
-                    if (active) {
-                        const float delta = ctl->desc_q[st].delta, scale = ctl->desc_q[st].scale;
-                        const uint64_t stored2 = pk2(stored, stored);
-                        const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
-                        uint64_t ctr = ctl->desc_q[st].ctr0 + K_GROUP * (uint64_t)rec.x;
-                        OutT* out = packed + ctl->desc_q[st].quad0 + rec.x;
-                        if (full) {
+            k += NW;
+            while (k >= nf) {
+                k -= nf;
+                ++it;
+            }
+        }
+        return;
+    }
+
+    for (; it < n_my;) {
+        const uint32_t round = fdiv(it, p.by_kq);
+        const uint32_t st = it - round * KQ;
+        if (!__all_sync(0xFFFFFFFFu, s_wait_chunk(&ctl->full_q[st], round & 1u, &ctl->desc_q[st].seq, it, p, ctl))) break;
+        const uint32_t nslots = ctl->desc_q[st].nslots;
+        if (k * 32u < nslots) {
+            const uint32_t sl = k * 32u + lane;
+            uint32_t rec = 0u;
+            if (sl < nslots) rec = table[sl];
+            const uint32_t rows = (rec >> 13) & 15u;
+            const bool active = rows != 0u;
+            const uint32_t which = (rec >> 17) & 3u;
+            const uint32_t quad = rec & 0x1FFFu;
+            const unsigned char* xs = ring_q + (size_t)st * stage_bytes + ((size_t)quad << QSHIFT);
+            const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
+            uint64_t vxy[P2], vzw[P2];
+            s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
+            const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
+            const float stored = Elem<LT>::round(mean);
+            if (active) {
+                const float delta = ctl->desc_q[st].delta, scale = ctl->desc_q[st].scale;
+                const uint64_t stored2 = pk2(stored, stored);
+                const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
+                uint64_t ctr = ctl->desc_q[st].ctr0 + K_GROUP * (uint64_t)quad;
+                OutT* out = packed + ctl->desc_q[st].quad0 + quad;
+                if (full) {
 #pragma unroll
-                            for (int r = 0; r < P2; ++r) {
-                                *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
-                                out += W4;
-                                ctr += p.rng_row_step;
-                            }
-                        } else {
-#pragma unroll
-                            for (int r = 0; r < P2; ++r) {
-                                if ((uint32_t)r < rows) {
-                                    *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
-                                    out += W4;
-                                    ctr += p.rng_row_step;
-                                }
-                            }
-                        }
+                    for (int r = 0; r < P2; ++r) {
+                        *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
+                        out += W4;
+                        ctr += p.rng_row_step;
                     }
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    if (atomicAdd(&ctl->done_q[st], 1u) == nf - 1u) {
-                        ctl->done_q[st] = 0u;
-                        __threadfence_block();
-                        mbar_arrive(&ctl->empty_q[st]);
+                } else {
+#pragma unroll
+                    for (int r = 0; r < P2; ++r) {
+                        if ((uint32_t)r < rows) {
+                            *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
+                            out += W4;
+                            ctr += p.rng_row_step;
+                        }
                     }
                 }
             }
         }
+        __syncwarp();
+        if (lane == 0) {
+            if (atomicAdd(&ctl->done_q[st], 1u) == nf - 1u) {
+                ctl->done_q[st] = 0u;
+                __threadfence_block();
+                mbar_arrive(&ctl->empty_q[st]);
+                atomicAdd(&ctl->q_closed, 1u);
+            }
+        }
         k += NW;
-        while (k >= 2u * nf) {
-            k -= 2u * nf;
-            ++step;
+        while (k >= nf) {
+            k -= nf;
+            ++it;
         }
     }
 }
@@ -684,38 +693,36 @@ inline div_status plan_staged(const div_desc* d, const Shape& s, SPlan* out) {
     if (G > bands_up) G = bands_up;
     pl.G = G;
     pl.slots = G * pl.spb;
-    if (pl.slots > 4096u) return DIV_ERR_PARAM;
+    if (pl.slots > 4096u || G * s.Wb > 4096u) return DIV_ERR_PARAM;         // widths of the strip table's fields
     pl.nf = (pl.slots + 31u) / 32u;
     pl.chunk_elems = pl.uniform ? G * s.B * s.W : (G / s.Hb) * s.HW;
-    if (pl.chunk_elems >= (1u << 20)) return DIV_ERR_PARAM;
+    if (pl.chunk_elems >= (1u << 15)) return DIV_ERR_PARAM;
     pl.chunks_per_sample = (pl.bands_per_sample + G - 1u) / G;
     pl.stage_bytes = (pl.chunk_elems * sx + 127u) & ~127u;
-    const uint32_t fixed = ((pl.slots * 8u + 15u) & ~15u) + (uint32_t)sizeof(SCtl) + 256u;
-    if ((uint32_t)di.smem_optin < fixed + 4u * pl.stage_bytes + 1024u) return DIV_ERR_PARAM;
-    uint32_t stages = ((uint32_t)di.smem_optin - 1024u - fixed) / pl.stage_bytes;
+    // shared memory: the two rings, the strip table, the control block; as many stages as fit, half of them
+    // (rounded down) for the quantise ring, whose copies come from the L2 and land sooner
+    const uint32_t fixed = ((pl.slots * 4u + 15u) & ~15u) + (uint32_t)sizeof(SCtl) + 16u;
+    if ((uint32_t)di.smem_optin < fixed + 4u * pl.stage_bytes) return DIV_ERR_PARAM;
+    uint32_t stages = ((uint32_t)di.smem_optin - fixed) / pl.stage_bytes;
     if (stages > 2u * S_MAX_STAGES) stages = 2u * S_MAX_STAGES;
-    uint32_t kq = (stages * 3u + 4u) / 8u;
-    if (kq < 2u) kq = 2u;
-    if (kq > (uint32_t)S_MAX_STAGES) kq = S_MAX_STAGES;
-    uint32_t kr = stages - kq;
-    if (kr > (uint32_t)S_MAX_STAGES) kr = S_MAX_STAGES;
-    if (kr < 2u) return DIV_ERR_PARAM;
+    const uint32_t kq = stages / 2u, kr = stages - kq;
     pl.kr = kr;
     pl.kq = kq;
     pl.smem_bytes = (int32_t)((kr + kq) * pl.stage_bytes + fixed);
     pl.total_chunks = (uint64_t)pl.chunks_per_sample * s.N;
-    // lag: at least a whole sample (see the progress argument at the top), and about DIVK_S_LAG_BYTES of x
-    const uint64_t chunk_bytes = (uint64_t)pl.chunk_elems * sx;
-    uint64_t lag = (DIVK_S_LAG_BYTES + chunk_bytes - 1) / chunk_bytes;
-    if (lag < (uint64_t)pl.chunks_per_sample + 2u) lag = (uint64_t)pl.chunks_per_sample + 2u;
-    if (lag > pl.total_chunks) lag = pl.total_chunks;     // a tensor smaller than the span: reduce everything, then quantise
     uint64_t grid = (uint64_t)di.sms;
     if (grid > pl.total_chunks) grid = pl.total_chunks;
     pl.grid = (int32_t)grid;
     pl.threads = S_THREADS;
-    // chunk indices and the claim counter are 32-bit on the device (every CTA overshoots by two claims)
-    if (pl.total_chunks + lag + 2u * grid >= (1ull << 30)) return DIV_ERR_PARAM;
-    pl.lag_chunks = (uint32_t)lag;
+    if (pl.total_chunks + grid >= (1ull << 30)) return DIV_ERR_PARAM;        // chunk indices are 32-bit on the device
+    // lag in rounds of `grid` chunks: the rounds a sample can spread over plus one (see the progress argument at
+    // the top), and about DIVK_S_LAG_BYTES of x
+    const uint64_t round_bytes = (uint64_t)pl.chunk_elems * sx * grid;
+    uint64_t lag = (DIVK_S_LAG_BYTES + round_bytes - 1) / round_bytes;
+    const uint64_t need = ((uint64_t)pl.chunks_per_sample - 1u + grid - 1u) / grid + 1u;
+    if (lag < need) lag = need;
+    if (lag >= (1ull << 20)) return DIV_ERR_PARAM;
+    pl.lag_steps = (uint32_t)lag;
     *out = pl;
     return DIV_OK;
 }
