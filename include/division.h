@@ -93,9 +93,10 @@ typedef struct div_layout {
 typedef struct div_plan {
     int32_t fused;          /* for W%4==0, B in {4,8}, Q in {2,4,8}, one launch:
                                6: x read from HBM once and re-read from L2 a little later, both reads staged through
-                                  shared-memory rings by bulk copies (staged kernel; first choice from 40 MB up);
-                               2: chunks wait in a shared-memory ring (strip ring kernel; first choice below 40 MB);
-                               3: as 6, with plain global loads (lagged kernel; next in line after 6 and 2);
+                                  shared-memory rings by bulk copies (staged kernel; first choice from 56 MB up
+                                  with B = 8);
+                               3: as 6, with plain global loads (lagged kernel; first choice from 20 MB up);
+                               2: chunks wait in a shared-memory ring (strip ring kernel; first choice below 20 MB);
                                4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
                                   at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;

@@ -159,11 +159,15 @@ div_status compress_two_pass(const div_desc* d, const Shape& s, const div_layout
 // ------------------------------------------------------------------------------------------
 constexpr int DEC_QPT = 4;
 
-// Which compress kernels run a descriptor.  Large maps go to the staged kernel (both reads of x staged through
-// shared memory by bulk copies), small ones to the strip ring kernel (shorter start-up); the lagged kernel
-// and the general kernels take what those two cannot.
+// Which compress kernels run a descriptor.  Measured on the ResNet / WRN / DenseNet-shaped maps: from about
+// 56 MB up with 8 x 8 blocks the staged kernel is fastest (both reads of x staged through shared memory by bulk
+// copies), from about 20 MB up the lagged kernel (plain loads, several bands per lane, cheap for small strips),
+// below that the strip ring kernel (shorter start-up); the general kernels take what those three cannot.
 bool prefer_staged(const div_desc* d, const Shape& s) {
-    return s.total * dtype_bytes(d->x_dtype) >= (40ull << 20);
+    return s.B == 8 && s.total * dtype_bytes(d->x_dtype) >= (56ull << 20);
+}
+bool prefer_lagged(const div_desc* d, const Shape& s) {
+    return s.total * dtype_bytes(d->x_dtype) >= (20ull << 20);
 }
 
 struct Choice {
@@ -187,12 +191,11 @@ void choose_compress(const div_desc* d, const Shape& s, uint32_t flags, Choice* 
     const bool may_staged = !(flags & DIV_FLAG_NO_STAGED_KERNEL);
     const bool may_lag = !(flags & DIV_FLAG_NO_LAGGED_KERNEL);
     const bool may_strip = !(flags & DIV_FLAG_NO_STRIP_KERNEL);
-    const bool big = prefer_staged(d, s);
-    if (may_staged && big && plan_staged(d, s, &c->sp) == DIV_OK) {
+    if (may_staged && prefer_staged(d, s) && plan_staged(d, s, &c->sp) == DIV_OK) {
         c->code = 6;
         return;
     }
-    if (may_lag && big && plan_lagged(d, s, &c->lp) == DIV_OK) {
+    if (may_lag && prefer_lagged(d, s) && plan_lagged(d, s, &c->lp) == DIV_OK) {
         c->code = 3;
         return;
     }

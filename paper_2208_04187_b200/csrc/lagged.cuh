@@ -332,6 +332,8 @@ lagged_kernel(const LParams p) {
             }
             const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
             const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+            // bar.warp.sync orders the other lanes' stores of low-frequency values before lane 0's release below
+            __syncwarp();
             if (lane == 0) {
                 uint32_t* slot = p.ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
                 red_max_relaxed(slot + 0, kmin);

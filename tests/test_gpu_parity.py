@@ -182,8 +182,9 @@ def test_fused_path_is_taken_where_expected():
     assert fused[(2, 2, 70, 70, 64, 2, "f32", "f32")] == 0        # block wider than a warp
     for spec in synth.config2() + synth.config1() + synth.config3():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
-        big = spec.numel * (4 if spec.x_dtype == "f32" else 2) >= 40 * 2 ** 20
-        assert binding.div_plan_query(d).fused == ((6 if big else 2) if spec.w % 4 == 0 else 4), spec.label()
+        nbytes = spec.numel * (4 if spec.x_dtype == "f32" else 2)
+        first = 6 if (nbytes >= 56 * 2 ** 20 and spec.block == 8) else (3 if nbytes >= 20 * 2 ** 20 else 2)
+        assert binding.div_plan_query(d).fused == (first if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
         assert binding.div_plan_query(d, STAGED).fused == (6 if spec.w % 4 == 0 else 4), spec.label()
