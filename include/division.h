@@ -40,7 +40,8 @@
  * Ownership and behaviour common to all entry points:
  *   - every pointer named *_dev is DEVICE memory owned by the caller, 16-byte aligned;
  *     descriptors and layouts are HOST memory;
- *   - the library allocates nothing and keeps no state between calls;
+ *   - the library allocates nothing and keeps no state between calls (one exception, documented there:
+ *     div_compress_static works in a fixed array inside the library);
  *   - div_compress / div_decompress only enqueue work on the given CUDA stream (a cudaStream_t
  *     passed as void*; NULL is the default stream) and return; errors that can be seen on the
  *     host are returned at once and nothing is launched;
@@ -175,18 +176,29 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
  *   DIV_ERR_CUDA      when the address of the array cannot be obtained on the current device.
  *
  * Things to know:
- *   - the first call on each device looks up the device address of the array (a host-side runtime query
- *     with that device current); make that first call outside any stream capture;
+ *   - every call asks the CUDA runtime for the device address of the array (a host-side query with the
+ *     current device; the first one on a device may make the runtime load the library's code onto it): make
+ *     the first call on each device outside any stream capture;
  *   - all calls on one device share the one array.  Each call clears the part it uses before its kernel
  *     runs (on the given stream), so earlier contents do not matter, but two calls whose work overlaps on
  *     the GPU (different streams, or different host threads without ordering between their streams) race
  *     on it and produce wrong output.  Keep calls on a device ordered one after the other;
  *   - the output is byte-for-byte what div_compress writes for the same arguments;
- *   - the device-side status word (see div_read_device_status) lives in the array and is not exposed.
+ *   - the device-side status word (a bounded wait that ran out, see div_read_device_status) lives in the
+ *     array: read it with div_read_static_status before the next call on that device overwrites it.
  */
 #define DIV_STATIC_MAX_SAMPLES 1024
 div_status div_compress_static(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,
                                uint64_t seed, void* cuda_stream);
+
+/*
+ * Device-side status of the last div_compress_static on the current device (no counterpart in the paper):
+ * what div_read_device_status reports for a caller-owned workspace, read from the library's fixed array.
+ * Synchronises the stream, copies one word back; allocates nothing.  *out_status is DIV_OK or
+ * DIV_ERR_TIMEOUT (the blob of that call is then unspecified: compress again, e.g. with div_compress_ex and
+ * DIV_FLAG_FORCE_TWO_PASS, whose kernels have no device-side waits).  Host-blocking.
+ */
+div_status div_read_static_status(void* cuda_stream, int32_t* out_status);
 
 /*
  * Decompress (Sec. 4.2; Algorithm 1, backward loop): x_hat = UpSampling(H^L) + Delta*V^H + delta,

@@ -14,8 +14,11 @@ operators that cache a packed 1-bit mask instead of an activation map.
 
 What is compressed: CUDA tensors of dtype fp32 / bf16 with 3 or 4 dimensions (Minibatch x Channel x N and
 Minibatch x Channel x N x N) and at least `min_elems` elements that are not leaves requiring grad (parameters).
-Everything else autograd saves is kept as it is.  All calls go to the current stream; one cache object must not be
-used from two streams at once (its scratch buffer is shared by its calls).
+Everything else autograd saves is kept as it is.  All calls go to the current stream.  Every compress call gets a
+scratch slice of its own (a few KB, from an arena that is reused from one forward pass to the next), so calls on
+different streams do not meet in it, and its device-side status word stays readable: the first decompress of a
+backward pass (or `check()`) reads all of them back in one copy and raises if a bounded wait inside a compress
+kernel ran out, instead of handing a corrupt activation map to the backward pass.
 """
 from __future__ import annotations
 
@@ -60,7 +63,9 @@ class DivisionCache:
         self.maps = 0
         self.records = []           # (seed, shape, dtype name) per compressed map, in forward order
         self._descs = {}
-        self._workspace = None
+        self._arena = []            # [tensor, bytes used] scratch chunks; a compress call takes a slice of its own
+        self._slices = []           # (chunk index, byte offset) of the slices handed out since __enter__
+        self._checked = 0           # slices whose status word has been read back
         self._seen = {}
         self._hooks = None
 
@@ -74,10 +79,37 @@ class DivisionCache:
             self._descs[key] = (desc, layout)
         return key, self._descs[key]
 
+    ARENA_CHUNK_BYTES = 1 << 20
+
     def _scratch(self, nbytes, device):
-        if self._workspace is None or self._workspace.numel() < nbytes or self._workspace.device != device:
-            self._workspace = torch.empty(max(int(nbytes), 1), dtype=torch.uint8, device=device)
-        return self._workspace
+        """A scratch slice of its own for one compress call (256-byte aligned, never shared with another call)."""
+        need = (int(nbytes) + 255) // 256 * 256
+        for ci, entry in enumerate(self._arena):
+            chunk, used = entry
+            if chunk.device == device and used + need <= chunk.numel():
+                entry[1] = used + need
+                self._slices.append((ci, used))
+                return chunk[used:used + need]
+        chunk = torch.empty(max(self.ARENA_CHUNK_BYTES, need), dtype=torch.uint8, device=device)
+        self._arena.append([chunk, need])
+        self._slices.append((len(self._arena) - 1, 0))
+        return chunk[:need]
+
+    def check(self):
+        """Read back the device-side status words of the compress calls made since the last check (one gather per
+        arena chunk, host-blocking) and raise DivisionError if a bounded wait ran out in one of them."""
+        todo = self._slices[self._checked:]
+        self._checked = len(self._slices)
+        by_chunk = {}
+        for ci, off in todo:
+            by_chunk.setdefault(ci, []).append(off // 4)
+        for ci, words in by_chunk.items():
+            chunk = self._arena[ci][0]
+            idx = torch.tensor(words, dtype=torch.int64).to(chunk.device, non_blocking=True)
+            status = chunk.view(torch.int32).index_select(0, idx).cpu()
+            bad = status.nonzero()
+            if bad.numel():
+                raise binding.DivisionError(int(status[bad[0, 0]]), "div_compress (device side, seen by DivisionCache)")
 
     # -- hooks ------------------------------------------------------------------------------------------------
     def pack(self, t: torch.Tensor):
@@ -112,6 +144,8 @@ class DivisionCache:
     def unpack(self, h):
         if not isinstance(h, _Cached):
             return h
+        if self._checked < len(self._slices):
+            self.check()
         desc, _ = self._descs[h.codec_key]
         out = torch.empty(h.shape, dtype=h.dtype, device=h.blob.device)
         stream = binding.current_stream_handle()
@@ -122,6 +156,12 @@ class DivisionCache:
         return out
 
     def __enter__(self):
+        # the arena is reused: what the previous forward pass put there has been consumed by its kernels, which
+        # precede this pass's kernels on the stream
+        for entry in self._arena:
+            entry[1] = 0
+        self._slices = []
+        self._checked = 0
         self._hooks = torch.autograd.graph.saved_tensors_hooks(self.pack, self.unpack)
         self._hooks.__enter__()
         return self

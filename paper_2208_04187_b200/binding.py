@@ -24,7 +24,8 @@ DIV_FLAG_NO_STAGED_KERNEL = 32
 DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 
 EXPORTED_SYMBOLS = (
-    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_debug_compress_starved",
+    "div_compressed_bytes", "div_compress", "div_compress_ex", "div_compress_static", "div_read_static_status",
+    "div_debug_compress_starved",
     "div_decompress", "div_plan_query",
     "div_compressed_bytes_3d", "div_compress_3d", "div_decompress_3d",
     "div_mask_bytes", "div_relu_forward", "div_dropout_forward", "div_mask_backward",
@@ -82,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.div_compress_ex.restype = c_int32
         L.div_compress_static.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_void_p, c_size_t, c_uint64, c_void_p]
         L.div_compress_static.restype = c_int32
+        L.div_read_static_status.argtypes = [c_void_p, ctypes.POINTER(c_int32)]
+        L.div_read_static_status.restype = c_int32
         L.div_debug_compress_starved.argtypes = L.div_compress_ex.argtypes + [c_uint64]
         L.div_debug_compress_starved.restype = c_int32
         L.div_decompress.argtypes = [ctypes.POINTER(DivDesc), c_void_p, c_size_t, c_void_p, c_void_p]
@@ -168,6 +171,13 @@ def div_compress_static(desc: DivDesc, x_ptr: int, comp_ptr: int, comp_capacity:
     st = lib().div_compress_static(ctypes.byref(desc), c_void_p(x_ptr), c_void_p(comp_ptr), comp_capacity,
                                    c_uint64(seed & (2 ** 64 - 1)), c_void_p(stream))
     _check(st, "div_compress_static")
+
+
+def div_read_static_status(stream: int = 0) -> int:
+    """Device-side status of the last div_compress_static on the current device (DIV_OK or DIV_ERR_TIMEOUT)."""
+    out = c_int32(0)
+    _check(lib().div_read_static_status(c_void_p(stream), ctypes.byref(out)), "div_read_static_status")
+    return out.value
 
 
 def div_decompress(desc: DivDesc, comp_ptr: int, comp_bytes: int, xhat_ptr: int, stream: int = 0) -> None:

@@ -1,11 +1,10 @@
 // Host side of the C ABI declared in include/division.h: argument checks, byte-layout arithmetic,
-// kernel selection and launches.  Nothing here allocates device memory or keeps state.
+// kernel selection and launches.  Nothing here allocates device memory; the only device memory the library
+// owns is the fixed scratch array of div_compress_static.
 #include "../../include/division.h"
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
-
-#include <mutex>
 
 #include "common.cuh"
 #include "decompress.cuh"
@@ -472,28 +471,17 @@ constexpr size_t STATIC_WS_BYTES =
     (4ull * (divk::WS_HEADER_WORDS + (size_t)divk::WS_SLOT_WORDS * DIV_STATIC_MAX_SAMPLES) + 255ull) / 256ull * 256ull;
 static __device__ __align__(256) unsigned char g_static_workspace[STATIC_WS_BYTES];
 
-constexpr int STATIC_MAX_DEVICES = 64;
-std::mutex g_static_mutex;
-void* g_static_ptr[STATIC_MAX_DEVICES] = {};     // device address of the array, per device ordinal
-
 // Device address of g_static_workspace on the current device.  In host code the array's name is only a
-// handle for the runtime, not an address a kernel could use, so the address is asked for once per device.
+// handle for the runtime, not an address a kernel could use, so the address is asked for (a host-side
+// query, no allocation); asking on every call keeps the library free of cached pointers that a device reset
+// would leave dangling.
 div_status static_workspace_ptr(void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) {
         cudaGetLastError();
         return DIV_ERR_CUDA;
     }
-    std::lock_guard<std::mutex> lock(g_static_mutex);
-    if (!g_static_ptr[dev]) {
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) {
-            cudaGetLastError();
-            return DIV_ERR_CUDA;
-        }
-        g_static_ptr[dev] = ptr;
-    }
-    *out = g_static_ptr[dev];
+    *out = ptr;
     return DIV_OK;
 }
 
@@ -512,6 +500,14 @@ div_status div_compress_static(const div_desc* desc, const void* x_dev, void* co
     if (got != DIV_OK) return got;
     // same path as div_compress from here on (it clears the part of the scratch it uses on the stream)
     return div_compress_ex(desc, x_dev, comp_dev, comp_capacity, ws, STATIC_WS_BYTES, seed, cuda_stream, 0u);
+}
+
+div_status div_read_static_status(void* cuda_stream, int32_t* out_status) {
+    if (!out_status) return DIV_ERR_NULL;
+    void* ws = nullptr;
+    const div_status got = static_workspace_ptr(&ws);
+    if (got != DIV_OK) return got;
+    return div_read_device_status(ws, cuda_stream, out_status);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -116,3 +116,28 @@ def test_a_residual_network_trains_through_the_cache():
         den1 += float(p.grad.square().sum())
         den2 += float(r.grad.square().sum())
     assert num / (den1 * den2) ** 0.5 > 0.98
+
+
+def test_cache_reads_back_device_status_and_raises_on_a_recorded_timeout():
+    """Every compress call of the cache has a scratch slice of its own; the first decompress of the backward pass
+    reads their status words back.  A timeout is planted by hand in one slice (no kernel is made to wait)."""
+    x_np = synth.activation_map(4, 8, 32, 32, "bn", 5)
+    leaf = torch.from_numpy(x_np).cuda().requires_grad_(True)
+    with dv.DivisionCache(block=8, qbits=2, seed=1, min_elems=1) as cache:
+        a = Probe.apply(leaf * 1.0)
+        b = Probe.apply(a * 1.0)
+    assert cache.maps == 2 and len(cache._slices) == 2
+    assert cache._slices[0] != cache._slices[1]                 # no scratch is shared between the two calls
+    cache.check()                                               # both status words are DIV_OK
+    Probe.seen.clear()
+    b.sum().backward()
+    assert len(Probe.seen) == 2
+
+    with dv.DivisionCache(block=8, qbits=2, seed=1, min_elems=1) as cache2:
+        y = Probe.apply(leaf * 1.0)
+    ci, off = cache2._slices[0]
+    torch.cuda.synchronize()
+    cache2._arena[ci][0].view(torch.int32)[off // 4] = binding.DIV_ERR_TIMEOUT
+    with pytest.raises(binding.DivisionError) as err:
+        y.sum().backward()
+    assert err.value.status == binding.DIV_ERR_TIMEOUT

@@ -2,12 +2,12 @@
 
 Some users of this library run where a device allocation is off limits at the moment they compress (inside
 another framework's callback, with the memory budget already handed out, or in a loop that must not pay for
-a device-synchronising cudaMalloc).  For them the library carries its own fixed scratch array.  This test
-calls that entry point through the C ABI twice in a row and checks that each result equals, byte for byte,
-what the ordinary div_compress writes for the same input and seed (the bar of the other parity tests), and
-that the fixed array's stale contents from the first call do not leak into the second.
-
-The file name sorts last on purpose: a run that stops at the first failure has then run every other test.
+a device-synchronising cudaMalloc).  For them the library carries its own fixed scratch array.  These tests
+call that entry point through the C ABI several times in a row, on maps that take each of the single-launch
+compress kernels, and check every result against the CPU checker and, byte for byte, against what the
+ordinary div_compress writes for the same input and seed (the bar of the other parity tests): the fixed
+array's stale contents from one call (claim counters, arrival counts, published parameters) must not leak
+into the next.
 """
 import ctypes
 
@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import division_oracle as orc
 from paper_2208_04187_b200 import binding, build, synth
 
 pytestmark = pytest.mark.gpu
@@ -34,39 +35,86 @@ def _reference_blob(x, desc_args, seed):
     return codec, codec.blob.clone()
 
 
-def test_static_scratch_matches_div_compress_on_two_calls_in_a_row():
+def _sections(blob, lo):
+    return (blob[lo.lfc_off:lo.lfc_off + lo.lfc_bytes], blob[lo.packed_off:lo.packed_off + lo.packed_bytes],
+            blob[lo.stats_off:lo.stats_off + lo.stats_bytes])
+
+
+def _assert_equals_checker(blob, layout, x_np, block, qbits, seed, samples):
+    """The blob's sections for the given samples equal what the CPU checker computes for them."""
+    n, c, h, w = x_np.shape
+    host = blob.cpu().numpy()
+    lfc = host[layout.lfc_off:layout.lfc_off + layout.lfc_bytes].view("<f4")
+    words = host[layout.packed_off:layout.packed_off + layout.packed_bytes].view("<u4")
+    stats = host[layout.stats_off:layout.stats_off + layout.stats_bytes].view("<f4").reshape(-1, 2)
+    hb, wb = orc.grid_shape(h, w, block)
+    tps, wps = c * hb * wb, c * h * w * qbits // 32
+    for i in samples:
+        ref = orc.compress(x_np[i:i + 1], block, qbits, seed, first_sample=i)
+        np.testing.assert_array_equal(lfc[i * tps:(i + 1) * tps], ref.lfc.reshape(-1))
+        np.testing.assert_array_equal(stats[i], [ref.delta[0], ref.step[0]])
+        np.testing.assert_array_equal(words[i * wps:(i + 1) * wps], ref.words)
+
+
+def test_static_scratch_matches_the_checker_and_div_compress_on_calls_in_a_row():
     stream = binding.current_stream_handle()
-    # two different maps, so that the second call finds the first call's leftovers in the shared array
-    spec_a = synth.config0()[0]                                   # 8 x 64 x 32 x 32, strip ring kernel
-    xa = torch.from_numpy(synth.make_input(spec_a)).cuda()
-    xb = torch.from_numpy(synth.activation_map(5, 24, 14, 14, "relu", 4242)).cuda()   # general ring kernel
-    args_a = (*spec_a.shape, spec_a.block, spec_a.qbits)
-    args_b = (5, 24, 14, 14, 8, 2)
-    codec_a, want_a = _reference_blob(xa, args_a, seed=11)
-    codec_b, want_b = _reference_blob(xb, args_b, seed=12)
+    # four maps of different shapes, one per compress path that keeps state in the scratch, so that every call
+    # finds another kernel's leftovers in the shared array
+    cases = [
+        ("strip ring kernel", synth.make_input(synth.config0()[0]), 8, 2, 2),                      # 8 x 64 x 32 x 32
+        ("plane pair", synth.activation_map(5, 24, 14, 14, "relu", 4242), 8, 2, 4),
+        ("lagged kernel", synth.activation_map(8, 64, 112, 112, "relu", 4243), 8, 2, 3),             # 25.7 MB
+        ("staged kernel", synth.activation_map(20, 64, 112, 112, "relu", 4244), 8, 2, 6),            # 64.2 MB
+    ]
+    prepared = []
+    for name, x_np, block, qbits, plan_code in cases:
+        args = (*x_np.shape, block, qbits)
+        x = torch.from_numpy(x_np).cuda()
+        codec, want = _reference_blob(x, args, seed=11)
+        assert codec.plan().fused == plan_code, name
+        prepared.append((name, x_np, x, codec, want, block, qbits))
 
-    got_a = torch.full_like(want_a, 0xEE)
-    got_b = torch.full_like(want_b, 0xEE)
-    got_a2 = torch.full_like(want_a, 0xEE)
-    # back to back on one stream: a, b, a again
-    binding.div_compress_static(codec_a.desc, xa.data_ptr(), got_a.data_ptr(), got_a.numel(), 11, stream)
-    binding.div_compress_static(codec_b.desc, xb.data_ptr(), got_b.data_ptr(), got_b.numel(), 12, stream)
-    binding.div_compress_static(codec_a.desc, xa.data_ptr(), got_a2.data_ptr(), got_a2.numel(), 11, stream)
+    # back to back on one stream: every map, then every map again in reverse order
+    order = list(range(len(prepared))) + list(reversed(range(len(prepared))))
+    outputs = []
+    for i in order:
+        name, x_np, x, codec, want, block, qbits = prepared[i]
+        got = torch.full_like(want, 0xEE)
+        binding.div_compress_static(codec.desc, x.data_ptr(), got.data_ptr(), got.numel(), 11, stream)
+        outputs.append((i, got))
     torch.cuda.synchronize()
+    assert binding.div_read_static_status(stream) == binding.DIV_OK
 
-    def sections(blob, layout):
-        lo = layout
-        return (blob[lo.lfc_off:lo.lfc_off + lo.lfc_bytes], blob[lo.packed_off:lo.packed_off + lo.packed_bytes],
-                blob[lo.stats_off:lo.stats_off + lo.stats_bytes])
-
-    for got, want, codec in ((got_a, want_a, codec_a), (got_b, want_b, codec_b), (got_a2, want_a, codec_a)):
-        for g, w in zip(sections(got, codec.layout), sections(want, codec.layout)):
-            assert torch.equal(g, w)
+    for i, got in outputs:
+        name, x_np, x, codec, want, block, qbits = prepared[i]
+        for g, w in zip(_sections(got, codec.layout), _sections(want, codec.layout)):
+            assert torch.equal(g, w), name
+        n = x_np.shape[0]
+        _assert_equals_checker(got, codec.layout, x_np, block, qbits, 11, sorted({0, n // 2, n - 1}))
     # and the result decodes like any other blob
-    xhat = codec_a.decompress(blob=got_a2)
-    xref = codec_a.decompress(blob=want_a)
+    name, x_np, x, codec, want, block, qbits = prepared[0]
+    xhat = codec.decompress(blob=outputs[-1][1])
+    xref = codec.decompress(blob=want)
     torch.cuda.synchronize()
     assert torch.equal(xhat, xref)
+
+
+def test_static_status_word_is_readable_through_its_accessor():
+    """The device-side status of a static call (a bounded wait that ran out would show here) can be read without
+    knowing where the library keeps its array; bad arguments are refused."""
+    stream = binding.current_stream_handle()
+    spec = synth.config0()[0]
+    x_np = synth.make_input(spec)
+    x = torch.from_numpy(x_np).cuda()
+    codec = binding.Codec(*spec.shape, spec.block, spec.qbits)
+    got = torch.zeros_like(codec.blob)
+    binding.div_compress_static(codec.desc, x.data_ptr(), got.data_ptr(), got.numel(), 5, stream)
+    torch.cuda.synchronize()
+    assert binding.div_read_static_status(stream) == binding.DIV_OK
+    _assert_equals_checker(got, codec.layout, x_np, spec.block, spec.qbits, 5, range(spec.n))
+    out = ctypes.c_int32(-1)
+    assert binding.lib().div_read_static_status(None, None) == binding.DIV_ERR_NULL
+    assert binding.lib().div_read_static_status(ctypes.c_void_p(stream), ctypes.byref(out)) == binding.DIV_OK and out.value == 0
 
 
 def test_static_scratch_refuses_more_samples_than_it_has_slots_for():
