@@ -28,17 +28,26 @@ sys.path.insert(0, ROOT)
 METRIC = "compress+decompress GB/s of activation"
 UNIT = "GB/s"
 WORKLOAD = "config2: ResNet-50 ImageNet-shaped set, batch 64 fp32, B=8, Q=2, fp32 LFC (5 maps, 590 MB)"
+MIN_TIMED_MS = 1000.0        # device time the headline rests on (the timed loop of --steps steps is repeated)
+MAX_REPEATS = 2000
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes per launch of the dominant kernel (lagged compress kernel on the 64x64x112x112 map):
-# dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture, see profiles/.  Set to None whenever that
-# kernel changes after the capture.
-NCU_TRAFFIC_BYTES = 214285824      # 206828288 read + 7457536 written (profiles/lagged_kernel_and_decompress_quad_map_64x64x112x112.md)
-
-
-# The same for the per-plane strip kernel on that map (profiles/pg_strip_kernel_and_pg_decompress_quad_map_64x64x112x112.md).
-PG_NCU_TRAFFIC_BYTES = 221775104   # 205539328 read + 16235776 written
+# DRAM bytes per launch of profiled kernels come from profiles/traffic.json (written next to the ncu summaries):
+# each entry names the kernel, the map, dram__bytes_read.sum / dram__bytes_write.sum of one capture and the
+# SHA-256 of the kernel's source file at capture time.  An entry whose source has changed since is not used.
+def ncu_traffic(kernel: str, map_label: str):
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            table = json.load(f)
+        e = table[f"{kernel} on {map_label}"]
+        with open(os.path.join(ROOT, e["source"]), "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != e["source_sha256"]:
+                return None
+        return int(e["dram_bytes_read"]) + int(e["dram_bytes_write"])
+    except Exception:
+        return None
 
 
 def measured_peak():
@@ -141,8 +150,38 @@ def oracle_step(inputs):
 
 
 def cpu_threads_used() -> int:
-    # the checker is plain NumPy elementwise code: it runs on one thread
+    # the checker is plain NumPy elementwise code: one call runs on one thread
     return 1
+
+
+_POOL_INPUTS = None
+
+
+def _oracle_task(task):
+    """One (map, sample) unit of the workload in a worker process (inputs inherited by fork, not pickled)."""
+    from oracle import division_oracle as orc
+    m, i = task
+    spec, x = _POOL_INPUTS[m]
+    comp = orc.compress(x[i:i + 1], spec.block, spec.qbits, 0, spec.x_dtype, spec.lfc_dtype, first_sample=i)
+    orc.decompress(comp)
+    return x[i:i + 1].nbytes
+
+
+def time_oracle_all_cores(inputs):
+    """The checker as it stands, samples dealt to one worker process per host core (samples are independent units)."""
+    import multiprocessing as mp
+    global _POOL_INPUTS
+    _POOL_INPUTS = inputs
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    tasks = [(m, i) for m, (spec, x) in enumerate(inputs) for i in range(x.shape[0])]
+    tasks.sort(key=lambda t: -inputs[t[0]][1][t[1]:t[1] + 1].nbytes)          # large units first
+    with mp.get_context("fork").Pool(cores) as pool:
+        pool.map(_oracle_task, tasks[:cores])                                  # start-up and imports, untimed
+        t0 = time.perf_counter()
+        nbytes = sum(pool.map(_oracle_task, tasks, chunksize=1))
+        dt = time.perf_counter() - t0
+    _POOL_INPUTS = None
+    return nbytes / dt / 1e9, cores
 
 
 def time_oracle(steps: int, warmup: int, samples_per_map: int):
@@ -237,6 +276,73 @@ def measure_train_step(device, ev, barrier, batch=64, steps=3):
     return out
 
 
+def measure_configs(device, ev, barrier, configs, peak, names, dec_names):
+    """The other workload configurations (seeded synthetic maps shaped like the paper's ResNet-18 / WRN-28-10 /
+    DenseNet-121 activations): every tensor compressed and decompressed on its own, back-to-back calls between two
+    CUDA events.  A tensor smaller than the L2 rotates over a pool of copies larger than twice the L2, inputs and
+    outputs alike, so that no call finds its data there."""
+    import torch
+
+    from paper_2208_04187_b200 import binding, synth
+
+    L2_BYTES = 126 * 2 ** 20
+    out = {}
+    for cfg in configs:
+        rows = []
+        raw_total, c_total, d_total = 0, 0.0, 0.0
+        for spec in synth.config_specs(cfg):
+            x = torch.from_numpy(synth.make_input(spec))
+            if spec.x_dtype == "bf16":
+                x = x.view(torch.bfloat16)
+            x = x.to(device)
+            nbytes = x.numel() * x.element_size()
+            pool = 2 if nbytes > L2_BYTES else int(2 * L2_BYTES // nbytes) + 2
+            xs = [x] + [x.clone() for _ in range(pool - 1)]
+            outs = [torch.empty_like(x) for _ in range(pool)]
+            codec = binding.Codec(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype, device=device)
+            plan = codec.plan()
+            algo = int(codec.layout.raw_bytes) + int(codec.layout.closed_form_bytes)
+            reps = max(10, min(60, int(2e9 // algo)))
+            for k in range(3):
+                codec.compress(xs[k % pool], seed=0)
+                codec.decompress(out=outs[k % pool])
+            barrier()
+            a, b = ev(), ev()
+            a.record()
+            for k in range(reps):
+                codec.compress(xs[k % pool], seed=0)
+            b.record()
+            barrier()
+            c_us = a.elapsed_time(b) * 1e3 / reps
+            assert codec.device_status() == binding.DIV_OK
+            a, b = ev(), ev()
+            a.record()
+            for k in range(reps):
+                codec.decompress(out=outs[k % pool])
+            b.record()
+            barrier()
+            d_us = a.elapsed_time(b) * 1e3 / reps
+            rows.append({"map": "x".join(map(str, spec.shape)) + f" {spec.x_dtype} {spec.kind} B{spec.block} Q{spec.qbits}",
+                         "MB": round(nbytes / 1e6, 1), "pool": pool, "calls": reps,
+                         "compress_kernel": names[int(plan.fused)], "compress_us": round(c_us, 1),
+                         "compress_GBps": round(algo / c_us / 1e3, 1), "compress_frac": round(algo / c_us / 1e3 / peak, 3),
+                         "decompress_kernel": dec_names[int(plan.decompress_fast)], "decompress_us": round(d_us, 1),
+                         "decompress_GBps": round(algo / d_us / 1e3, 1), "decompress_frac": round(algo / d_us / 1e3 / peak, 3)})
+            raw_total += nbytes
+            c_total += c_us
+            d_total += d_us
+            del xs, outs, x, codec
+            torch.cuda.empty_cache()
+        out[f"config{cfg}"] = {"tensors": len(rows), "raw_MB": round(raw_total / 1e6, 1),
+                               "compress_us_sum": round(c_total, 1), "decompress_us_sum": round(d_total, 1),
+                               "GBps_of_activation": round(raw_total / (c_total + d_total) / 1e3, 1), "per_tensor": rows}
+    out["what"] = ("every tensor of the configuration on its own: back-to-back calls through the C ABI between two CUDA events, "
+                   "inputs and outputs rotating over a pool of copies > 2 x L2 where the tensor is smaller than the L2; us per call "
+                   "include the launch cost a caller sees (the smallest maps are bound by it); GBps = algorithmic bytes "
+                   "(raw + closed-form compressed) / time; frac = GBps / measured HBM peak")
+    return out
+
+
 # ----------------------------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------------------------
@@ -259,8 +365,9 @@ def run_ours(args):
     build.build()
     binding.lib()
 
-    kernel_names_all = {5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel", 3: "lagged_kernel",
-                        2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
+    kernel_names_all = {6: "staged_kernel", 5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel",
+                        3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
+    dec_names_all = {1: "decompress_quad_kernel", 2: "decompress_flat_kernel", 3: "decompress_line_kernel", 0: "decompress_general_kernel"}
     specs = synth.config_specs(2)
     if args.maps:
         specs = [specs[int(i)] for i in args.maps.split(",")]
@@ -304,14 +411,21 @@ def run_ours(args):
     sampler.start()
     time.sleep(0.25)
     barrier()
-    # the timed region: exactly args.steps steps between two events, nothing else on the stream
-    t_start, t_end = ev(), ev()
-    t_start.record()
-    for k in range(args.steps):
-        step()
-    t_end.record()
-    barrier()
-    total_ms = t_start.elapsed_time(t_end)
+    # the timed region: exactly args.steps steps between two events, nothing else on the stream; repeated (same
+    # number of steps each time) until at least MIN_TIMED_MS of device time has been measured, so that a short
+    # --steps still rests on a second of samples.  ms_per_step is the median over the repeats.
+    rep_ms = []
+    while True:
+        t_start, t_end = ev(), ev()
+        t_start.record()
+        for k in range(args.steps):
+            step()
+        t_end.record()
+        barrier()
+        rep_ms.append(t_start.elapsed_time(t_end))
+        if sum(rep_ms) >= MIN_TIMED_MS or len(rep_ms) >= MAX_REPEATS:
+            break
+    total_ms = statistics.median(rep_ms)
     # a second, instrumented pass for the per-call figures (an event pair around every call costs a few us per
     # call, which is why it is kept out of the timed region above)
     rec_steps = max(3, min(args.steps, 100))
@@ -325,6 +439,23 @@ def run_ours(args):
                for i in range(len(codecs))]
     dec_ms = [statistics.mean(records[k][1][i][0].elapsed_time(records[k][1][i][1]) for k in range(rec_steps))
               for i in range(len(codecs))]
+
+    # ---- the dominant kernel alone: back-to-back launches of the slowest compress call, two input buffers
+    # ---- alternating (410 MB, far above the L2), no events between the calls
+    dom = max(range(len(specs)), key=lambda i: comp_ms[i])
+    alt = torch.empty_like(dev_x[dom]).copy_(dev_x[dom])
+    dom_n = max(20, min(args.steps, 100))
+    for k in range(3):
+        codecs[dom].compress(alt if k % 2 else dev_x[dom], seed=0, flags=args.compress_flags)
+    barrier()
+    d0, d1 = ev(), ev()
+    d0.record()
+    for k in range(dom_n):
+        codecs[dom].compress(alt if k % 2 else dev_x[dom], seed=0, flags=args.compress_flags)
+    d1.record()
+    barrier()
+    dom_ms = d0.elapsed_time(d1) / dom_n
+    del alt
 
     # ---- end to end through the C ABI with host buffers: H2D of x, compress, decompress, D2H of x_hat ----
     host_out = [torch.empty_like(h).pin_memory() for h in host_x]
@@ -431,7 +562,7 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "kernel": pg_names[int(pg_plans[pg_dom].fused)] + " on " +
                          "x".join(map(str, specs[pg_dom].shape)), "achieved": pg_dom_gbs, "peak": pg_peak,
                          "unit": "GB/s", "frac": pg_dom_gbs / pg_peak, "peak_kind": f"of {pg_peak_kind}",
-                         "traffic": PG_NCU_TRAFFIC_BYTES if specs[pg_dom].shape == (64, 64, 112, 112) else None,
+                         "traffic": ncu_traffic(pg_names[int(pg_plans[pg_dom].fused)], "x".join(map(str, specs[pg_dom].shape))),
                          "algorithmic_bytes_per_launch": pg_algo[pg_dom]},
         }
 
@@ -570,6 +701,18 @@ def run_ours(args):
                    "peak_kind": f"of {pk3_kind}", "gpu_launches": 3 * (n3 + 3)}
         del pairs3, blob3, ws3
 
+    # ---- the other workload configurations, tensor by tensor ----
+    other_configs = None
+    if args.configs and not args.maps:
+        dev_x.clear()                   # hand the benchmark's device buffers back first
+        dev_out.clear()
+        for c in codecs:
+            c.blob = c.workspace = None
+        torch.cuda.empty_cache()
+        cfg_peak, _ = measured_peak()
+        other_configs = measure_configs(device, ev, barrier, [int(c) for c in args.configs.split(",")], cfg_peak,
+                                        kernel_names_all, dec_names_all)
+
     # ---- Algorithm 1 around a synthetic ResNet-50 step: activation memory (after forward - after backward) and
     # ---- forward+backward time, plain autograd against the cache (B=8, Q=2; ReLU with packed masks) ----
     train_step = None
@@ -596,22 +739,25 @@ def run_ours(args):
     algo_bytes = [int(c.layout.raw_bytes) + int(c.layout.closed_form_bytes) for c in codecs]
     comp_gbs = sum(algo_bytes) / (sum(comp_ms) * 1e-3) / 1e9
     dec_gbs = sum(algo_bytes) / (sum(dec_ms) * 1e-3) / 1e9
-    kernel_names = {5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel", 3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
+    kernel_names = kernel_names_all
     per_map = [{"map": "x".join(map(str, s.shape)), "compress_kernel": kernel_names[int(p.fused)],
                 "compress_us": round(cm * 1e3, 2), "compress_GBps": round(b / cm / 1e6, 1),
                 "decompress_us": round(dm * 1e3, 2), "decompress_GBps": round(b / dm / 1e6, 1)}
                for s, p, cm, dm, b in zip(specs, plans, comp_ms, dec_ms, algo_bytes)]
-    # dominant kernel: the compress kernel of the largest map (largest share of the step's device time)
-    dom = max(range(len(specs)), key=lambda i: comp_ms[i])
-    dom_gbs = algo_bytes[dom] / (comp_ms[dom] * 1e-3) / 1e9
+    # dominant kernel: the compress kernel with the largest share of the step's device time, timed alone above
+    dom_gbs = algo_bytes[dom] / (dom_ms * 1e-3) / 1e9
 
     # CPU baseline: the checker on the whole workload once (after one warm-up on a slice)
     cpu = None
     if not args.no_cpu_baseline and world == 1:
+        inputs = [(sp, h.numpy()) for sp, h in zip(specs, host_x)]
         time_oracle(1, 0, 1)
-        gbs, _ = time_oracle(1, 0, 64)
-        cpu = {"value": gbs, "unit": UNIT, "cores": cpu_threads_used(), "kind": "oracle",
-               "sample": "the whole config-2 workload (5 maps, 64 samples each), one pass, NumPy checker as it stands"}
+        gbs1, _ = time_oracle(1, 0, 8)
+        gbs, cores = time_oracle_all_cores(inputs)
+        cpu = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "the whole config-2 workload (5 maps, 64 samples each), one pass, NumPy checker as it stands, "
+                         "samples dealt to one process per host core",
+               "single_thread": {"value": gbs1, "cores": cpu_threads_used(), "sample": "first 8 samples of each of the 5 maps"}}
 
     line = {
         "metric": METRIC, "value": job_bytes / (job_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -620,15 +766,20 @@ def run_ours(args):
         "config": {"workload": WORKLOAD + (f" [maps {args.maps} only]" if args.maps else ""), "maps": [m["map"] for m in per_map],
                    "l2": "working set 1.2 GB per step, every buffer touched once per step: far above the 126 MB L2",
                    "order": "compress maps 0..4, then decompress maps 0..4",
-                   "timing": f"value / ms_per_step: {args.steps} steps between two CUDA events, nothing else on the stream; "
-                             f"per_map and roofline: a second pass of {rec_steps} steps with an event pair around every call",
+                   "timing": f"value / ms_per_step: median of {len(rep_ms)} repeats of {args.steps} steps between two CUDA events "
+                             f"(min {min(rep_ms) / args.steps:.4f} ms, max {max(rep_ms) / args.steps:.4f} ms per step), nothing else on the "
+                             f"stream; per_map: a second pass of {rec_steps} steps with an event pair around every call; roofline: the "
+                             "dominant kernel alone, back to back",
+                   "ms_per_step_min": min(rep_ms) / args.steps, "ms_per_step_max": max(rep_ms) / args.steps, "repeats": len(rep_ms),
                    "multi_gpu": "replicas only: each rank runs the same set on its own GPU, no collective",
                    "compression_ratio": raw_bytes / comp_bytes, "per_map": per_map},
         "roofline": {"bound": "hbm", "kernel": kernel_names[int(plans[dom].fused)] + " on " + per_map[dom]["map"] +
-                     " (CUDA events around the call on its stream, instrumented pass; the span includes the 2-us workspace clear)",
-                     "achieved": dom_gbs, "peak": peak, "unit": "GB/s", "frac": dom_gbs / peak,
+                     f" ({dom_n} back-to-back calls between two CUDA events on its stream, two inputs alternating; "
+                     "the span includes the 2-us workspace clear)",
+                     "achieved": dom_gbs, "peak": peak, "unit": "GB/s", "frac": dom_gbs / peak, "us_per_launch": dom_ms * 1e3,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": dom_gbs / NOMINAL_HBM_GBS,
-                     "traffic": NCU_TRAFFIC_BYTES, "algorithmic_bytes_per_launch": algo_bytes[dom]},
+                     "traffic": ncu_traffic(kernel_names[int(plans[dom].fused)], per_map[dom]["map"]),
+                     "algorithmic_bytes_per_launch": algo_bytes[dom]},
         "roofline_all_compress": {"bound": "hbm", "kernel": "all compress calls of the step", "achieved": comp_gbs,
                                   "peak": peak, "unit": "GB/s", "frac": comp_gbs / peak, "peak_kind": f"of {peak_kind}"},
         "roofline_all_decompress": {"bound": "hbm", "kernel": "all decompress calls of the step", "achieved": dec_gbs,
@@ -638,13 +789,14 @@ def run_ours(args):
         "mask_ops": mask_ops,
         "one_d": one_d,
         "three_d": three_d,
+        "configs": other_configs,
         "train_step": train_step,
         "e2e": {"value": raw_bytes * world / (e2e_job_ms * 1e-3) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": raw_bytes, "d2h_bytes_per_step": raw_bytes, "ms_per_step": e2e_job_ms,
                 "steps": e2e_steps,
                 "how": "pinned host buffers; per map: copy-in, compress, decompress, copy-out, on three streams ordered by "
                        "events so that the two PCIe directions and the kernels overlap"},
-        "gpu_launches": kernels_per_step * args.steps,
+        "gpu_launches": kernels_per_step * args.steps * len(rep_ms),
         "clocks": clocks,
     }
     print(json.dumps(line))
@@ -663,6 +815,8 @@ def main():
     ap.add_argument("--no-train-step", action="store_true", help="skip the ResNet-50 forward+backward memory / time measurement")
     ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D and 3-D maps")
     ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
+    ap.add_argument("--configs", default="0,1,3,4",
+                    help="other workload configurations to time tensor by tensor (empty: none); config 2 is the headline")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")
     ap.add_argument("--compress-flags", type=int, default=0,
                     help="DIV_FLAG_* bits passed to div_compress_ex (profiling aid: 4 = strip ring kernel instead of the lagged one)")

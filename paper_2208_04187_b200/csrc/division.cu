@@ -329,16 +329,25 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
     if ((s.total * (uint64_t)desc->qbits) % 32u != 0 &&
         cudaMemsetAsync(blob + lo.packed_off + lo.packed_bytes - 4, 0, 4, stream) != cudaSuccess)
         return DIV_ERR_CUDA;
-    Choice ch;
-    choose_compress(desc, s, flags, &ch);
-    switch (ch.code) {
-        case 5: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream);
-        case 6: return compress_staged(desc, s, lo, ch.sp, x_dev, blob, ws, seed, stream);
-        case 3: return compress_lagged(desc, s, lo, ch.lp, x_dev, blob, ws, seed, stream);
-        case 2: return compress_fused_v(desc, s, lo, ch.vp, x_dev, blob, ws, seed, stream);
-        case 4: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream);
-        case 1: return compress_fused(desc, s, lo, ch.fp, x_dev, blob, ws, seed, stream);
-        default: break;
+    // The single-launch kernels need all their CTAs resident, so they are launched cooperatively; where the
+    // device refuses such a launch (fewer SMs visible to the process than the device reports, for instance) the
+    // next kernel in line takes the descriptor: nothing has been enqueued by the refused launch.
+    for (uint32_t f = flags;;) {
+        Choice ch;
+        choose_compress(desc, s, f, &ch);
+        div_status r = DIV_OK;
+        uint32_t drop = 0;
+        switch (ch.code) {
+            case 5: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream);
+            case 6: r = compress_staged(desc, s, lo, ch.sp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STAGED_KERNEL; break;
+            case 3: r = compress_lagged(desc, s, lo, ch.lp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_LAGGED_KERNEL; break;
+            case 2: r = compress_fused_v(desc, s, lo, ch.vp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STRIP_KERNEL; break;
+            case 4: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream);
+            case 1: r = compress_fused(desc, s, lo, ch.fp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_FORCE_TWO_PASS; break;
+            default: return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
+        }
+        if (r != DIV_ERR_CUDA) return r;
+        f |= drop;
     }
     return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
 }

@@ -22,6 +22,8 @@
 // certain that all CTAs are resident (no grid-wide barrier is used).
 #pragma once
 
+#include <atomic>
+
 #include "../../include/division.h"
 #include "common.cuh"
 #include "twopass.cuh"   // Shape
@@ -441,21 +443,61 @@ struct DeviceInfo {
     int sms;
     int smem_optin;
     bool ok;
+    int dev;
 };
+
+// What the planners need to know about a device is asked from the runtime once per device and kept (a few words
+// of host memory per device ordinal): a call of div_compress then costs one cudaGetDevice instead of attribute,
+// occupancy and function-attribute queries.  Ordinals of DEVICE_CACHE_SLOTS or above are served without the cache.
+constexpr int DEVICE_CACHE_SLOTS = 64;
 inline DeviceInfo device_info() {
-    DeviceInfo di = {0, 0, false};
+    static std::atomic<int> cached_sms[DEVICE_CACHE_SLOTS];
+    static std::atomic<int> cached_smem[DEVICE_CACHE_SLOTS];
+    DeviceInfo di = {0, 0, false, -1};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
         return di;
+    }
+    di.dev = dev;
+    const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
+    if (slot) {
+        di.sms = cached_sms[dev].load(std::memory_order_acquire);
+        di.smem_optin = cached_smem[dev].load(std::memory_order_acquire);
+        if (di.sms > 0 && di.smem_optin > 0) {
+            di.ok = true;
+            return di;
+        }
     }
     if (cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&di.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
         cudaGetLastError();
         return di;
     }
+    if (slot) {
+        cached_smem[dev].store(di.smem_optin, std::memory_order_release);
+        cached_sms[dev].store(di.sms, std::memory_order_release);
+    }
     di.ok = true;
     return di;
+}
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize of one kernel: set once per device and size, not once per launch.
+// `seen` is the per-kernel table of the largest size already set on each device.
+inline bool ensure_dynamic_smem(const void* kern, int bytes, std::atomic<int>* seen) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
+    if (slot && seen[dev].load(std::memory_order_acquire) >= bytes) return true;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    if (slot) seen[dev].store(bytes, std::memory_order_release);
+    return true;
 }
 
 // Decide whether and how the fused kernel runs a descriptor.  DIV_OK: plan filled in.
@@ -528,10 +570,8 @@ inline div_status plan_fused(const div_desc* d, const Shape& s, FusedPlan* out) 
 template <typename XT, typename LT, int Q, int P2>
 inline div_status launch_fused(const FusedParams& prm, cudaStream_t st) {
     auto kern = fused_compress_kernel<XT, LT, Q, P2>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, prm.pl.smem_bytes) != cudaSuccess) {
-        cudaGetLastError();
-        return DIV_ERR_CUDA;
-    }
+    static std::atomic<int> smem_set[DEVICE_CACHE_SLOTS];
+    if (!ensure_dynamic_smem((const void*)kern, prm.pl.smem_bytes, smem_set)) return DIV_ERR_CUDA;
     void* args[] = {(void*)&prm};
     if (cudaLaunchCooperativeKernel((const void*)kern, dim3(prm.pl.grid), dim3(prm.pl.threads), args,
                                     (size_t)prm.pl.smem_bytes, st) != cudaSuccess) {

@@ -455,24 +455,35 @@ lagged_kernel(const LParams p) {
 // host side
 // ------------------------------------------------------------------------------------------------
 template <typename XT, typename LT, int Q, int P2>
-inline div_status l_occupancy(int* ctas_per_sm) {
+inline div_status l_occupancy(int dev, int* ctas_per_sm) {
+    // resident CTAs per SM of this instance: asked once per device
+    static std::atomic<int> cached[DEVICE_CACHE_SLOTS];
+    const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
+    if (slot) {
+        const int c = cached[dev].load(std::memory_order_acquire);
+        if (c > 0) {
+            *ctas_per_sm = c;
+            return DIV_OK;
+        }
+    }
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, lagged_kernel<XT, LT, Q, P2>, L_THREADS, 0) != cudaSuccess) {
         cudaGetLastError();
         return DIV_ERR_CUDA;
     }
+    if (slot && *ctas_per_sm > 0) cached[dev].store(*ctas_per_sm, std::memory_order_release);
     return DIV_OK;
 }
 
 template <typename XT, typename LT>
-inline div_status l_occupancy_q(int qbits, uint32_t p2, int* out) {
+inline div_status l_occupancy_q(int dev, int qbits, uint32_t p2, int* out) {
     if (p2 == 8) {
-        if (qbits == 2) return l_occupancy<XT, LT, 2, 8>(out);
-        if (qbits == 4) return l_occupancy<XT, LT, 4, 8>(out);
-        if (qbits == 8) return l_occupancy<XT, LT, 8, 8>(out);
+        if (qbits == 2) return l_occupancy<XT, LT, 2, 8>(dev, out);
+        if (qbits == 4) return l_occupancy<XT, LT, 4, 8>(dev, out);
+        if (qbits == 8) return l_occupancy<XT, LT, 8, 8>(dev, out);
     } else if (p2 == 4) {
-        if (qbits == 2) return l_occupancy<XT, LT, 2, 4>(out);
-        if (qbits == 4) return l_occupancy<XT, LT, 4, 4>(out);
-        if (qbits == 8) return l_occupancy<XT, LT, 8, 4>(out);
+        if (qbits == 2) return l_occupancy<XT, LT, 2, 4>(dev, out);
+        if (qbits == 4) return l_occupancy<XT, LT, 4, 4>(dev, out);
+        if (qbits == 8) return l_occupancy<XT, LT, 8, 4>(dev, out);
     }
     return DIV_ERR_PARAM;
 }
@@ -506,9 +517,9 @@ inline div_status plan_lagged(const div_desc* d, const Shape& s, LPlan* out) {
     int cps = 0;
     div_status st;
     if (d->x_dtype == DIV_F32)
-        st = d->lfc_dtype == DIV_F32 ? l_occupancy_q<float, float>(d->qbits, s.P2, &cps) : l_occupancy_q<float, bf16>(d->qbits, s.P2, &cps);
+        st = d->lfc_dtype == DIV_F32 ? l_occupancy_q<float, float>(di.dev, d->qbits, s.P2, &cps) : l_occupancy_q<float, bf16>(di.dev, d->qbits, s.P2, &cps);
     else
-        st = d->lfc_dtype == DIV_F32 ? l_occupancy_q<bf16, float>(d->qbits, s.P2, &cps) : l_occupancy_q<bf16, bf16>(d->qbits, s.P2, &cps);
+        st = d->lfc_dtype == DIV_F32 ? l_occupancy_q<bf16, float>(di.dev, d->qbits, s.P2, &cps) : l_occupancy_q<bf16, bf16>(di.dev, d->qbits, s.P2, &cps);
     if (st != DIV_OK) return st;
     if (cps < 1) return DIV_ERR_CUDA;
     pl.ctas_per_sm = cps;

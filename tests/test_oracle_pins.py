@@ -63,6 +63,44 @@ def test_lfc_tail_tiles_average_in_bounds_elements(shape, block):
     np.testing.assert_allclose(got, ref, rtol=0, atol=1e-6 * np.abs(x).max())
 
 
+def test_block_sum_order_is_columns_first_pairwise_trees():
+    """The block sum is a balanced pairwise tree down the rows of every tile column, then the same tree across
+    the column sums.  One 8 x 8 tile on which this order, the rows-first order and a running sum round
+    differently in fp32 (2^24 + 1 is not representable and rounds to 2^24); the expected value is worked out
+    by hand, not by the checker:
+        column 0 = (1, 2^24, 1, -2^24, 0, ...):  (1 + 2^24) + (1 - 2^24) = 2^24 + (-16777215) = 1
+        column 1 = (1, 0,    1, 0,     0, ...):  (1 + 0) + (1 + 0) = 2
+        across the columns: (1 + 2) + 0 + ... = 3, mean = 3 / 64        (the exact sum is 4)."""
+    big = np.float32(2.0 ** 24)
+    tile = np.zeros((8, 8), dtype=np.float32)
+    tile[:4, 0] = [1, big, 1, -big]
+    tile[:4, 1] = [1, 0, 1, 0]
+    got = orc.lfc_mean_f32(tile[None, None], 8)
+    assert got.shape == (1, 1, 1, 1)
+    assert got[0, 0, 0, 0] == np.float32(3.0 / 64.0)
+
+    def tree(values):
+        v = [np.float32(a) for a in values]
+        while len(v) > 1:
+            v = [np.float32(v[i] + v[i + 1]) for i in range(0, len(v), 2)]
+        return v[0]
+
+    # the other orders give other numbers on this tile, so the pin tells them apart
+    rows_first = tree([tree(tile[r, :]) for r in range(8)])          # (2 + 2^24) + (2 - 2^24) = 4
+    running = np.float32(0)
+    for v in tile.T.reshape(-1):                                     # column by column, one element after the other
+        running = np.float32(running + v)                            # ((1 + 2^24) + 1) - 2^24 = 0, then + 2
+    assert rows_first == np.float32(4) and running == np.float32(2)
+    assert float(tile.astype(np.float64).sum()) == 4.0
+    # the same tile inside a larger map, next to ordinary tiles, and as a partial tile (5 in-bounds rows)
+    x = bn_map((1, 2, 16, 16), 21)
+    x[0, 1, 8:16, 0:8] = tile
+    assert orc.lfc_mean_f32(x, 8)[0, 1, 1, 0] == np.float32(3.0 / 64.0)
+    part = np.zeros((1, 1, 13, 8), dtype=np.float32)
+    part[0, 0, 8:13, :] = tile[:5]
+    assert orc.lfc_mean_f32(part, 8)[0, 0, 1, 0] == np.float32(np.float32(3.0) / np.float32(40.0))
+
+
 def test_side_shorter_than_block_gives_1x1_plane_mean():
     """Sec. 4.1 footnote: N < B makes the low-frequency map Minibatch x Channel x 1 x 1."""
     x = bn_map((3, 5, 7, 7), 13)
