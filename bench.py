@@ -365,7 +365,7 @@ def run_ours(args):
     build.build()
     binding.lib()
 
-    kernel_names_all = {6: "staged_kernel", 5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel",
+    kernel_names_all = {7: "plane_fused_kernel", 6: "staged_kernel", 5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel",
                         3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
     dec_names_all = {1: "decompress_quad_kernel", 2: "decompress_flat_kernel", 3: "decompress_line_kernel", 0: "decompress_general_kernel"}
     specs = synth.config_specs(2)
@@ -378,7 +378,7 @@ def run_ours(args):
     plans = [c.plan(args.compress_flags) for c in codecs]
     raw_bytes = sum(int(c.layout.raw_bytes) for c in codecs)
     comp_bytes = sum(int(c.layout.closed_form_bytes) for c in codecs)
-    kernels_per_step = sum((2 if p.fused in (0, 4, 5) else 1) + 1 for p in plans)
+    kernels_per_step = sum((2 if p.fused in (0, 4, 5) else 1) + 1 for p in plans)      # compress launches + one decompress launch
     torch.cuda.synchronize()
 
     def step(record=None):
@@ -423,7 +423,7 @@ def run_ours(args):
         t_end.record()
         barrier()
         rep_ms.append(t_start.elapsed_time(t_end))
-        if sum(rep_ms) >= MIN_TIMED_MS or len(rep_ms) >= MAX_REPEATS:
+        if sum(rep_ms) >= MIN_TIMED_MS or len(rep_ms) >= args.max_repeats:
             break
     total_ms = statistics.median(rep_ms)
     # a second, instrumented pass for the per-call figures (an event pair around every call costs a few us per
@@ -815,6 +815,8 @@ def main():
     ap.add_argument("--no-train-step", action="store_true", help="skip the ResNet-50 forward+backward memory / time measurement")
     ap.add_argument("--no-one-d", action="store_true", help="skip the timing of the 1-D and 3-D maps")
     ap.add_argument("--no-masks", action="store_true", help="skip the timing of the ReLU / dropout mask operators")
+    ap.add_argument("--max-repeats", type=int, default=MAX_REPEATS,
+                    help="upper bound on the repeats of the timed loop (1 for a short run under a profiler)")
     ap.add_argument("--configs", default="0,1,3,4",
                     help="other workload configurations to time tensor by tensor (empty: none); config 2 is the headline")
     ap.add_argument("--maps", default="", help="comma-separated indices of the config-2 maps to run (profiling aid)")

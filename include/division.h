@@ -98,8 +98,11 @@ typedef struct div_plan {
                                   with B = 8);
                                3: as 6, with plain global loads (lagged kernel; first choice from 20 MB up);
                                2: chunks wait in a shared-memory ring (strip ring kernel; first choice below 20 MB);
-                               4: two launches for small planes of any width (tile side 4, 8 or 16 after padding,
-                                  at most 32 lanes per plane row, Q in {2,4,8}); the second read comes from L2;
+                               7: small planes of any width (tile side 4, 8 or 16 after padding, at most 32 lanes per
+                                  plane row, Q in {2,4,8}) in one launch: a CTA owns a run of planes of one sample,
+                                  joins the sample's other CTAs through an arrival count and quantises the same
+                                  planes (second read from L1 / L2); taken when all its CTAs can be resident;
+                               4: the same in two launches;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;
                                5: 1-D maps (h == 1; the appendix on 1D and 3D activation maps), W%4==0, B a power of two
                                   in [4,128], Q in {2,4,8}: two launches, the second read comes from L2 */
@@ -124,6 +127,7 @@ typedef struct div_plan {
 #define DIV_FLAG_NO_PLANE_KERNELS 8u /* never take the small-plane pair of kernels          */
 #define DIV_FLAG_NO_LINE_KERNELS 16u /* never take the pair of kernels for 1-D maps          */
 #define DIV_FLAG_NO_STAGED_KERNEL 32u/* never take the staged (bulk-copy rings) kernel       */
+#define DIV_FLAG_TWO_LAUNCH_PLANES 64u /* small planes: the pair of kernels, not the fused one */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:
@@ -211,12 +215,12 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                           void* xhat_dev, void* cuda_stream);
 
 /*
- * Test hook for the bounded waits of the single-launch compress kernels (plan codes 2, 3 and 6): runs the
+ * Test hook for the bounded waits of the single-launch compress kernels (plan codes 2, 3, 6 and 7): runs the
  * kernel div_compress_ex would run, but tells it to wait for a number of arrivals per sample that is never
  * reached, with `timeout_ns` (at most 100 ms) as the limit of every wait.  The kernel must give up, record
  * DIV_ERR_TIMEOUT in the workspace status word (read it with div_read_device_status) and return; the blob's
- * contents are then unspecified.  The first of the strip ring, lagged and staged kernels that the flags allow
- * and the descriptor fits is taken; DIV_ERR_PARAM when there is none.
+ * contents are then unspecified.  The first of the strip ring, lagged, staged and fused small-plane
+ * kernels that the flags allow and the descriptor fits is taken; DIV_ERR_PARAM when there is none.
  * Arguments as for div_compress_ex.  No counterpart in the paper.
  */
 div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, void* comp_dev, size_t comp_capacity,

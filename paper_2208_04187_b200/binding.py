@@ -21,6 +21,7 @@ DIV_FLAG_NO_LAGGED_KERNEL = 4
 DIV_FLAG_NO_PLANE_KERNELS = 8
 DIV_FLAG_NO_LINE_KERNELS = 16
 DIV_FLAG_NO_STAGED_KERNEL = 32
+DIV_FLAG_TWO_LAUNCH_PLANES = 64
 DTYPE_CODES = {"f32": DIV_F32, "bf16": DIV_BF16}
 
 EXPORTED_SYMBOLS = (

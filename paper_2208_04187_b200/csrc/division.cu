@@ -26,7 +26,8 @@ typedef __nv_bfloat16 bf16;
 
 constexpr uint64_t SECTION_ALIGN = 128;
 constexpr uint32_t DIV_FLAG_ALL = DIV_FLAG_FORCE_TWO_PASS | DIV_FLAG_NO_STRIP_KERNEL | DIV_FLAG_NO_LAGGED_KERNEL |
-                                  DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_NO_LINE_KERNELS | DIV_FLAG_NO_STAGED_KERNEL;
+                                  DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_NO_LINE_KERNELS | DIV_FLAG_NO_STAGED_KERNEL |
+                                  DIV_FLAG_TWO_LAUNCH_PLANES;
 
 inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
 inline uint32_t dtype_bytes(int32_t dt) { return dt == DIV_F32 ? 4u : 2u; }
@@ -176,6 +177,7 @@ struct Choice {
     LPlan lp;
     VPlan vp;
     PlaneGeom pg;
+    PlaneFusedPlan pf;
     FusedPlan fp;
 };
 
@@ -211,7 +213,7 @@ void choose_compress(const div_desc* d, const Shape& s, uint32_t flags, Choice* 
         return;
     }
     if (!(flags & DIV_FLAG_NO_PLANE_KERNELS) && plan_planes(d, s, &c->pg)) {
-        c->code = 4;
+        c->code = (!(flags & DIV_FLAG_TWO_LAUNCH_PLANES) && plane_fused_applies(d, s, c->pg, &c->pf)) ? 7 : 4;
         return;
     }
     if (plan_fused(d, s, &c->fp) == DIV_OK) c->code = 1;
@@ -289,6 +291,12 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
         out->smem_bytes = ch.vp.smem_bytes;
         out->chunk_elems = ch.vp.chunk_elems;
         out->chunks_per_sample = ch.vp.chunks_per_sample;
+    } else if (ch.code == 7) {
+        out->grid = (int32_t)(ch.pf.ctas_per_sample * s.N);
+        out->threads = 256;
+        out->smem_bytes = (int32_t)ch.pf.smem;
+        out->chunk_elems = (int64_t)ch.pf.ppc * s.HW;
+        out->chunks_per_sample = ch.pf.ctas_per_sample;
     } else if (ch.code == 4) {
         out->grid = (int32_t)((ch.pg.qps + 256 * PLANE_QPT - 1) / (256 * PLANE_QPT) * s.N);
         out->threads = 256;
@@ -342,7 +350,8 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
             case 6: r = compress_staged(desc, s, lo, ch.sp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STAGED_KERNEL; break;
             case 3: r = compress_lagged(desc, s, lo, ch.lp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_LAGGED_KERNEL; break;
             case 2: r = compress_fused_v(desc, s, lo, ch.vp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STRIP_KERNEL; break;
-            case 4: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream);
+            case 7: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream, true);
+            case 4: return compress_planes(desc, s, lo, ch.pg, x_dev, blob, ws, seed, stream, false);
             case 1: r = compress_fused(desc, s, lo, ch.fp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_FORCE_TWO_PASS; break;
             default: return compress_two_pass(desc, s, lo, x_dev, blob, ws, seed, stream);
         }
@@ -380,6 +389,10 @@ div_status div_debug_compress_starved(const div_desc* desc, const void* x_dev, v
     if (!(flags & DIV_FLAG_NO_STAGED_KERNEL)) {
         SPlan sp;
         if (plan_staged(desc, s, &sp) == DIV_OK) return compress_staged(desc, s, lo, sp, x_dev, blob, ws, seed, stream, never, timeout_ns);
+    }
+    if (!(flags & (DIV_FLAG_NO_PLANE_KERNELS | DIV_FLAG_TWO_LAUNCH_PLANES))) {
+        PlaneGeom pg;
+        if (plan_planes(desc, s, &pg)) return compress_planes(desc, s, lo, pg, x_dev, blob, ws, seed, stream, true, never, timeout_ns);
     }
     return DIV_ERR_PARAM;
 }

@@ -483,20 +483,31 @@ inline DeviceInfo device_info() {
 }
 
 // cudaFuncAttributeMaxDynamicSharedMemorySize of one kernel: set once per device and size, not once per launch.
-// `seen` is the per-kernel table of the largest size already set on each device.
-inline bool ensure_dynamic_smem(const void* kern, int bytes, std::atomic<int>* seen) {
+// `seen` is the per-kernel table of what has been set on each device; an entry also names the kernel it is
+// about, so that a table shared by accident (two copies of the library in one process) is never trusted for
+// another copy's kernel.
+struct SmemSeen {
+    std::atomic<const void*> fn;
+    std::atomic<int> bytes;
+};
+inline bool ensure_dynamic_smem(const void* kern, int bytes, SmemSeen* seen) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) {
         cudaGetLastError();
         return false;
     }
     const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
-    if (slot && seen[dev].load(std::memory_order_acquire) >= bytes) return true;
+    if (slot && seen[dev].fn.load(std::memory_order_acquire) == kern && seen[dev].bytes.load(std::memory_order_acquire) >= bytes)
+        return true;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
         cudaGetLastError();
         return false;
     }
-    if (slot) seen[dev].store(bytes, std::memory_order_release);
+    if (slot) {
+        seen[dev].fn.store(nullptr, std::memory_order_release);
+        seen[dev].bytes.store(bytes, std::memory_order_release);
+        seen[dev].fn.store(kern, std::memory_order_release);
+    }
     return true;
 }
 
@@ -570,7 +581,7 @@ inline div_status plan_fused(const div_desc* d, const Shape& s, FusedPlan* out) 
 template <typename XT, typename LT, int Q, int P2>
 inline div_status launch_fused(const FusedParams& prm, cudaStream_t st) {
     auto kern = fused_compress_kernel<XT, LT, Q, P2>;
-    static std::atomic<int> smem_set[DEVICE_CACHE_SLOTS];
+    static SmemSeen smem_set[DEVICE_CACHE_SLOTS];
     if (!ensure_dynamic_smem((const void*)kern, prm.pl.smem_bytes, smem_set)) return DIV_ERR_CUDA;
     void* args[] = {(void*)&prm};
     if (cudaLaunchCooperativeKernel((const void*)kern, dim3(prm.pl.grid), dim3(prm.pl.threads), args,

@@ -705,7 +705,7 @@ inline div_status plan_v(const div_desc* d, const Shape& s, VPlan* out) {
 template <typename XT, typename LT, int Q, int P2>
 inline div_status launch_v(const VParams& prm, cudaStream_t st) {
     auto kern = fused_v_kernel<XT, LT, Q, P2>;
-    static std::atomic<int> smem_set[DEVICE_CACHE_SLOTS];
+    static SmemSeen smem_set[DEVICE_CACHE_SLOTS];
     if (!ensure_dynamic_smem((const void*)kern, prm.pl.smem_bytes, smem_set)) return DIV_ERR_CUDA;
     void* args[] = {(void*)&prm};
     if (cudaLaunchCooperativeKernel((const void*)kern, dim3(prm.pl.grid), dim3(prm.pl.threads), args,

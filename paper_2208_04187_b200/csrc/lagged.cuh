@@ -457,10 +457,11 @@ lagged_kernel(const LParams p) {
 template <typename XT, typename LT, int Q, int P2>
 inline div_status l_occupancy(int dev, int* ctas_per_sm) {
     // resident CTAs per SM of this instance: asked once per device
-    static std::atomic<int> cached[DEVICE_CACHE_SLOTS];
+    static SmemSeen cached[DEVICE_CACHE_SLOTS];          // .bytes holds the count
+    const void* kern = (const void*)lagged_kernel<XT, LT, Q, P2>;
     const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
-    if (slot) {
-        const int c = cached[dev].load(std::memory_order_acquire);
+    if (slot && cached[dev].fn.load(std::memory_order_acquire) == kern) {
+        const int c = cached[dev].bytes.load(std::memory_order_acquire);
         if (c > 0) {
             *ctas_per_sm = c;
             return DIV_OK;
@@ -470,7 +471,11 @@ inline div_status l_occupancy(int dev, int* ctas_per_sm) {
         cudaGetLastError();
         return DIV_ERR_CUDA;
     }
-    if (slot && *ctas_per_sm > 0) cached[dev].store(*ctas_per_sm, std::memory_order_release);
+    if (slot && *ctas_per_sm > 0) {
+        cached[dev].fn.store(nullptr, std::memory_order_release);
+        cached[dev].bytes.store(*ctas_per_sm, std::memory_order_release);
+        cached[dev].fn.store(kern, std::memory_order_release);
+    }
     return DIV_OK;
 }
 

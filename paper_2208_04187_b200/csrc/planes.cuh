@@ -1,7 +1,8 @@
 // Compress kernels for maps with small planes whose width is not a multiple of 4 (the 14 x 14 and
 // 7 x 7 maps of the ImageNet networks): DIVISION Sec. 4.1; Algorithm 1, forward loop.
 //
-// Two launches, no dependency inside a kernel:
+// plane_fused_kernel does both halves in one launch (see there); where its CTAs cannot all be resident the pair
+// below runs instead.  Two launches, no dependency inside a kernel:
 //   plane_stats_kernel   block means in the fixed summation order, stored low-frequency values,
 //                        residual extremes -> per-sample min / max keys in the scratch slots;
 //   plane_quant_kernel   Eq. 9 with stochastic rounding and packing, 4 consecutive elements per step.
@@ -149,6 +150,171 @@ plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const u
     }
 }
 
+// One launch for both halves.  CTA (b, n) owns the planes [b * ppc, (b + 1) * ppc) of sample n (ppc a multiple of 4
+// and of the planes a warp takes at once, so that its elements are a whole number of quads):
+//   1. block means, stored low-frequency values (also kept in shared memory) and residual extremes of its
+//      planes, exactly as plane_stats_kernel; the CTA's extremes are folded into the sample's slot (two
+//      reductions without an answer), then, behind a release fence, the CTA is counted as arrived;
+//   2. thread 0 waits (bounded) until all CTAs of the sample have arrived and derives (delta, Delta, scale);
+//   3. Eq. 9 and packing of the same planes as plane_quant_kernel, x read a second time (it is still in this
+//      SM's L1 or in the L2), the low-frequency values from shared memory.
+// The launch is cooperative so that the CTAs a wait depends on are resident; no grid-wide barrier is used.
+struct PlaneFused {
+    uint32_t ppc;                 // planes per CTA
+    uint32_t ctas_per_sample;
+    uint64_t timeout_ns;
+    uint32_t expected;            // arrivals that complete a sample (a test may ask for an unreachable count)
+};
+
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(256)
+plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, void* __restrict__ packed_v,
+                   float* __restrict__ stats, PlaneGeom g, PlaneFused f, uint64_t seed) {
+    typedef typename PackedUnit<Q>::type OutT;
+    extern __shared__ uint32_t plane_smem[];
+    uint16_t* tile_of = reinterpret_cast<uint16_t*>(plane_smem);          // position inside a plane -> tile inside the plane
+    float* lfc_s = reinterpret_cast<float*>(plane_smem + g.table_words);  // stored low-frequency values of this CTA's planes
+    __shared__ uint32_t s_kmin, s_kmax, s_delta, s_scale, s_ok;
+    const uint32_t n = blockIdx.y;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t plane0 = blockIdx.x * f.ppc;
+    const uint32_t nplanes = plane0 < g.C ? min(f.ppc, g.C - plane0) : 0u;
+    for (uint32_t idx = threadIdx.x; idx < g.HW; idx += 256u) {
+        const uint32_t h = fdiv(idx, g.by_w), w = idx - h * g.W;
+        tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * g.Wb + fdiv(w, g.by_b));
+    }
+    if (threadIdx.x == 0) {
+        s_kmin = 0;
+        s_kmax = 0;
+        s_ok = 0;
+    }
+    __syncthreads();
+
+    // ---------------- half 1: a lane owns one tile column of one plane ----------------
+    {
+        const uint32_t pl_local = lane / g.lanes_per_plane;
+        const uint32_t lw = lane - pl_local * g.lanes_per_plane;
+        const uint32_t bw = lw / P2, cw = lw % P2;
+        const uint32_t cols = (bw < g.Wb) ? min(g.B, g.W - bw * g.B) : 0u;
+        const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
+        const uint32_t col = bw * g.B + cw;
+        float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+        for (uint32_t pp = warp * g.planes_per_warp; pp < nplanes; pp += 8u * g.planes_per_warp) {
+            const uint32_t pl = pp + pl_local;                       // plane inside the CTA's run
+            const bool ok = lane_ok && pl < nplanes;
+            const XT* xp = x + ((size_t)n * g.C + plane0 + (ok ? pl : 0u)) * g.HW + (ok ? col : 0u);
+            LT* lp = lfc + ((size_t)n * g.C + plane0 + (ok ? pl : 0u)) * g.TPP + (ok ? bw : 0u);
+            for (uint32_t bh = 0; bh < g.Hb; ++bh) {
+                const uint32_t rows = min(g.B, g.H - bh * g.B);
+                float v[P2];
+#pragma unroll
+                for (int r = 0; r < P2; ++r) v[r] = (ok && (uint32_t)r < rows) ? Elem<XT>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0.f;
+                float sum = tree8<P2>(v);
+#pragma unroll
+                for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+                float mean = 0.f;
+                if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
+                mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
+                const float stored = Elem<LT>::round(mean);
+                if (ok) {
+                    if (cw == 0) {
+                        Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
+                        lfc_s[pl * g.TPP + bh * g.Wb + bw] = stored;
+                    }
+                    float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+#pragma unroll
+                    for (int r = 0; r < P2; ++r) {
+                        if ((uint32_t)r < rows) {
+                            blo = fminf(blo, v[r]);
+                            bhi = fmaxf(bhi, v[r]);
+                        }
+                    }
+                    lo = fminf(lo, __fsub_rn(blo, stored));
+                    hi = fmaxf(hi, __fsub_rn(bhi, stored));
+                }
+            }
+        }
+        const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
+        const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+        if (lane == 0) {
+            atomicMax(&s_kmin, kmin);
+            atomicMax(&s_kmax, kmax);
+        }
+    }
+    __syncthreads();
+
+    // ---------------- the sample's extremes: fold, count, wait for the other CTAs of the sample ----------------
+    if (threadIdx.x == 0) {
+        uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+        if (nplanes) {
+            red_max_relaxed(slot + 0, s_kmin);
+            red_max_relaxed(slot + 1, s_kmax);
+        }
+        fence_acq_rel_gpu();
+        asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(slot + 2), "r"(1u) : "memory");
+        uint32_t polls = 0;
+        uint64_t t0 = 0;
+        bool ok = true;
+        while (ld_acquire_u32(slot + 2) != f.expected) {
+            if ((++polls & 7u) == 0) {
+                const uint64_t tn = now_ns();
+                if (t0 == 0) t0 = tn;
+                if (ld_relaxed_u32(ws) != 0u || tn - t0 > f.timeout_ns) {
+                    atomicCAS(ws, 0u, (uint32_t)DIV_ERR_TIMEOUT);
+                    atomicCAS(ws + 1, 0u, n + 1u);
+                    ok = false;
+                    break;
+                }
+            }
+            __nanosleep(100);
+        }
+        if (ok) {
+            const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
+            if (blockIdx.x == 0) {
+                stats[2 * (size_t)n + 0] = qp.delta;
+                stats[2 * (size_t)n + 1] = qp.step;
+            }
+            s_delta = __float_as_uint(qp.delta);
+            s_scale = __float_as_uint(qp.scale);
+            s_ok = 1;
+        }
+    }
+    __syncthreads();
+    if (!s_ok || nplanes == 0) return;
+
+    // ---------------- half 2: a thread per 4 consecutive elements of the CTA's planes ----------------
+    const float delta = __uint_as_float(s_delta), scale = __uint_as_float(s_scale);
+    const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
+    const uint64_t base = rng_sample_base(seed, n);
+    const uint64_t sample_quad0 = (uint64_t)n * g.qps;
+    const XT* x_n = x + (size_t)n * g.CHW;
+    OutT* packed = reinterpret_cast<OutT*>(packed_v);
+    const uint32_t qa = (plane0 * g.HW) >> 2, qb = ((plane0 + nplanes) * g.HW) >> 2;     // this CTA's quads [qa, qb)
+    for (uint32_t q = qa + threadIdx.x; q < qb; q += 256u) {
+        uint64_t xy, zw;
+        StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy, zw);
+        const uint32_t plane = fdiv(q * 4u, g.by_hw);
+        uint32_t rem = q * 4u - plane * g.HW;
+        const float* lfc_p = lfc_s + (plane - plane0) * g.TPP;
+        float lf[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            lf[i] = lfc_p[tile_of[rem]];
+            if (++rem == g.HW) {
+                rem = 0;
+                lfc_p += g.TPP;
+            }
+        }
+        constexpr float qmax = (float)((1 << Q) - 1);
+        const uint64_t z = rng_group(base, q);
+        uint32_t b0, b1, b2, b3;
+        quant2(xy, pk2(lf[0], lf[1]), delta2, scale2, qmax, (uint32_t)z, b0, b1);
+        quant2(zw, pk2(lf[2], lf[3]), delta2, scale2, qmax, (uint32_t)(z >> 32), b2, b3);
+        constexpr uint32_t BIAS = QUANT2_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
+        packed[sample_quad0 + q] = (OutT)(b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -177,11 +343,126 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
     return true;
 }
 
+// resident CTAs per SM of one instance of the fused kernel with `smem` bytes of dynamic shared memory (asked
+// once per device and size)
+template <typename XT, typename LT, int Q, int P2>
+inline int plane_fused_occupancy(int dev, size_t smem) {
+    static SmemSeen cached[DEVICE_CACHE_SLOTS];          // .bytes holds (smem << 8) | count
+    const void* kern = (const void*)plane_fused_kernel<XT, LT, Q, P2>;
+    const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS && smem < (1u << 22);
+    if (slot && cached[dev].fn.load(std::memory_order_acquire) == kern) {
+        const int c = cached[dev].bytes.load(std::memory_order_acquire);
+        if ((size_t)(c >> 8) == smem && (c & 255) > 0) return c & 255;
+    }
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, plane_fused_kernel<XT, LT, Q, P2>, 256, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (slot && n > 0 && n < 256) {
+        cached[dev].fn.store(nullptr, std::memory_order_release);
+        cached[dev].bytes.store((int)((smem << 8) | (size_t)n), std::memory_order_release);
+        cached[dev].fn.store(kern, std::memory_order_release);
+    }
+    return n;
+}
+
+// How the single-launch form would run a descriptor; false when it does not apply (its CTAs could not all be resident)
+struct PlaneFusedPlan {
+    uint32_t ppc, ctas_per_sample;
+    size_t smem;
+};
+template <typename XT, typename LT, int Q, int P2>
+inline bool plan_plane_fused(const Shape& s, const PlaneGeom& g, const DeviceInfo& di, PlaneFusedPlan* out) {
+    // planes per CTA: a multiple of 4 (whole quads) and of the planes a warp takes at once; about 8 CTAs per SM in all
+    const uint32_t step = 4u / gcd_u32(4u, g.planes_per_warp) * g.planes_per_warp;
+    uint32_t want = (uint32_t)((8ull * di.sms + s.N - 1) / s.N);
+    if (want < 1) want = 1;
+    uint32_t ppc = ((s.C + want - 1) / want + step - 1) / step * step;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        const uint32_t cps = (s.C + ppc - 1) / ppc;
+        const size_t smem = 4ull * g.table_words + 4ull * ppc * s.TPP;
+        if (smem > 40000) return false;
+        const int occ = plane_fused_occupancy<XT, LT, Q, P2>(di.dev, smem);
+        if (occ < 1) return false;
+        if ((uint64_t)cps * s.N > (uint64_t)occ * di.sms) {
+            if (attempt) return false;
+            // fewer, larger CTAs so that all of them fit on the device at once
+            const uint64_t fit = ((uint64_t)occ * di.sms) / s.N;
+            if (fit < 1) return false;
+            ppc = (uint32_t)(((s.C + fit - 1) / fit + step - 1) / step * step);
+            continue;
+        }
+        out->ppc = ppc;
+        out->ctas_per_sample = cps;
+        out->smem = smem;
+        return true;
+    }
+    return false;
+}
+
+// launch of the single-launch form; false when it does not apply or the launch was refused
+template <typename XT, typename LT, int Q, int P2>
+inline bool launch_plane_fused(const Shape& s, const div_layout& lo, const PlaneGeom& g, const DeviceInfo& di, const void* x,
+                               uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, uint32_t expected, uint64_t timeout_ns) {
+    PlaneFusedPlan pf;
+    if (!plan_plane_fused<XT, LT, Q, P2>(s, g, di, &pf)) return false;
+    PlaneFused f;
+    f.ppc = pf.ppc;
+    f.ctas_per_sample = pf.ctas_per_sample;
+    f.timeout_ns = timeout_ns ? timeout_ns : 2000000000ull;
+    f.expected = expected ? expected : pf.ctas_per_sample;
+    const XT* xt = (const XT*)x;
+    LT* lfc = (LT*)(blob + lo.lfc_off);
+    void* packed = blob + lo.packed_off;
+    float* stats = (float*)(blob + lo.stats_off);
+    PlaneGeom gg = g;
+    void* args[] = {(void*)&xt, (void*)&lfc, (void*)&ws, (void*)&packed, (void*)&stats, (void*)&gg, (void*)&f, (void*)&seed};
+    if (cudaLaunchCooperativeKernel((const void*)plane_fused_kernel<XT, LT, Q, P2>, dim3(pf.ctas_per_sample, s.N), dim3(256), args,
+                                    pf.smem, st) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
+template <typename XT, typename LT>
+inline bool launch_plane_fused_q(int qbits, const Shape& s, const div_layout& lo, const PlaneGeom& g, const DeviceInfo& di,
+                                 const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, uint32_t expected,
+                                 uint64_t timeout_ns) {
+#define DIVK_PF(QQ, PP) launch_plane_fused<XT, LT, QQ, PP>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns)
+    switch (s.P2) {
+        case 4: return qbits == 2 ? DIVK_PF(2, 4) : qbits == 4 ? DIVK_PF(4, 4) : DIVK_PF(8, 4);
+        case 8: return qbits == 2 ? DIVK_PF(2, 8) : qbits == 4 ? DIVK_PF(4, 8) : DIVK_PF(8, 8);
+        case 16: return qbits == 2 ? DIVK_PF(2, 16) : qbits == 4 ? DIVK_PF(4, 16) : DIVK_PF(8, 16);
+    }
+#undef DIVK_PF
+    return false;
+}
+
+// would the single-launch form run this descriptor?  (fills grid / shared memory for div_plan_query)
+inline bool plane_fused_applies(const div_desc* d, const Shape& s, const PlaneGeom& g, PlaneFusedPlan* out) {
+    typedef __nv_bfloat16 bf16;
+    const DeviceInfo di = device_info();
+    if (!di.ok || di.sms < 1) return false;
+#define DIVK_PP(XT, LT, QQ, PP) plan_plane_fused<XT, LT, QQ, PP>(s, g, di, out)
+#define DIVK_PQ(XT, LT, PP) (d->qbits == 2 ? DIVK_PP(XT, LT, 2, PP) : d->qbits == 4 ? DIVK_PP(XT, LT, 4, PP) : DIVK_PP(XT, LT, 8, PP))
+#define DIVK_PT(XT, LT) (s.P2 == 4 ? DIVK_PQ(XT, LT, 4) : s.P2 == 8 ? DIVK_PQ(XT, LT, 8) : s.P2 == 16 ? DIVK_PQ(XT, LT, 16) : false)
+    if (d->x_dtype == DIV_F32) return d->lfc_dtype == DIV_F32 ? DIVK_PT(float, float) : DIVK_PT(float, bf16);
+    return d->lfc_dtype == DIV_F32 ? DIVK_PT(bf16, float) : DIVK_PT(bf16, bf16);
+#undef DIVK_PT
+#undef DIVK_PQ
+#undef DIVK_PP
+}
+
 template <typename XT, typename LT>
 inline div_status compress_planes_t(const div_desc* d, const Shape& s, const div_layout& lo, const PlaneGeom& g,
-                                    const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+                                    const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st,
+                                    bool allow_fused, uint32_t expected, uint64_t timeout_ns) {
     const DeviceInfo di = device_info();
     if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
+    if (allow_fused && launch_plane_fused_q<XT, LT>(d->qbits, s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns)) return DIV_OK;
+    if (expected) return DIV_ERR_PARAM;              // the test hook is about the single-launch form only
     // pass 1: enough CTAs per sample to fill the GPU a few times over, never more than there are warp passes
     uint32_t bx = (uint32_t)((8ull * di.sms + s.N - 1) / s.N);
     const uint32_t bx_max = (g.groups + 7u) / 8u;
@@ -212,14 +493,15 @@ inline div_status compress_planes_t(const div_desc* d, const Shape& s, const div
 }
 
 inline div_status compress_planes(const div_desc* d, const Shape& s, const div_layout& lo, const PlaneGeom& g,
-                                  const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+                                  const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st,
+                                  bool allow_fused = true, uint32_t expected = 0, uint64_t timeout_ns = 0) {
     typedef __nv_bfloat16 bf16;
     if (d->x_dtype == DIV_F32) {
-        if (d->lfc_dtype == DIV_F32) return compress_planes_t<float, float>(d, s, lo, g, x, blob, ws, seed, st);
-        return compress_planes_t<float, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+        if (d->lfc_dtype == DIV_F32) return compress_planes_t<float, float>(d, s, lo, g, x, blob, ws, seed, st, allow_fused, expected, timeout_ns);
+        return compress_planes_t<float, bf16>(d, s, lo, g, x, blob, ws, seed, st, allow_fused, expected, timeout_ns);
     }
-    if (d->lfc_dtype == DIV_F32) return compress_planes_t<bf16, float>(d, s, lo, g, x, blob, ws, seed, st);
-    return compress_planes_t<bf16, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+    if (d->lfc_dtype == DIV_F32) return compress_planes_t<bf16, float>(d, s, lo, g, x, blob, ws, seed, st, allow_fused, expected, timeout_ns);
+    return compress_planes_t<bf16, bf16>(d, s, lo, g, x, blob, ws, seed, st, allow_fused, expected, timeout_ns);
 }
 
 }  // namespace divk

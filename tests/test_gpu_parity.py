@@ -20,7 +20,8 @@ TWO_PASS = binding.DIV_FLAG_FORCE_TWO_PASS
 LAGGED = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_STAGED_KERNEL
 RING = binding.DIV_FLAG_NO_LAGGED_KERNEL | binding.DIV_FLAG_NO_STAGED_KERNEL
 STAGED = binding.DIV_FLAG_NO_STRIP_KERNEL | binding.DIV_FLAG_NO_LAGGED_KERNEL
-NO_SPECIAL = STAGED | binding.DIV_FLAG_NO_STAGED_KERNEL                     # planes pair, else general ring
+NO_SPECIAL = STAGED | binding.DIV_FLAG_NO_STAGED_KERNEL                     # small-plane kernels, else general ring
+PLANES_PAIR = NO_SPECIAL | binding.DIV_FLAG_TWO_LAUNCH_PLANES               # the small-plane pair instead of the fused kernel
 NO_STRIP = NO_SPECIAL | binding.DIV_FLAG_NO_PLANE_KERNELS                   # general ring, else two-pass
 
 
@@ -130,8 +131,8 @@ def small_input(n, c, h, w, x_dtype, seed):
 
 
 @pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(map(str, c)))
-@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS],
-                         ids=["default", "lagged", "staged", "planes", "general_ring", "two_pass"])
+@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS],
+                         ids=["default", "lagged", "staged", "planes", "planes_pair", "general_ring", "two_pass"])
 def test_small_cases_match_the_checker(case, flags):
     n, c, h, w, block, q, xd, ld = case
     x = small_input(n, c, h, w, xd, seed=n + c + h + w + block + q)
@@ -163,20 +164,21 @@ def test_fused_path_is_taken_where_expected():
             sx = 4 if xd == "f32" else 2
             b = min(block, max(h, w))
             aligned = (c * h * w * sx) % 16 == 0 and (h * w * sx) % 16 == 0 and (b * w * sx) % 16 == 0
-            assert staged[case] == (6 if aligned else (4 if planes_shape(case) else 1)), case
+            assert staged[case] == (6 if aligned else (7 if planes_shape(case) else 1)), case
         elif planes_shape(case):
-            assert fused[case] == 4 and lagged[case] == 4 and staged[case] == 4, case
+            assert fused[case] == 7 and lagged[case] == 7 and staged[case] == 7, case
+            assert binding.div_plan_query(binding.make_desc(*case), PLANES_PAIR).fused == 4, case
         else:
             assert fused[case] in (0, 1) and lagged[case] == fused[case] and staged[case] == fused[case], case
-        assert special[case] == (4 if planes_shape(case) else binding.div_plan_query(binding.make_desc(*case), NO_STRIP).fused), case
+        assert special[case] == (7 if planes_shape(case) else binding.div_plan_query(binding.make_desc(*case), NO_STRIP).fused), case
     assert sum(1 for c in SMALL if fused[c] == 2) >= 12
     assert sum(1 for c in SMALL if staged[c] == 6) >= 12
-    assert sum(1 for c in SMALL if fused[c] == 4) >= 5
-    assert sum(1 for c in SMALL if special[c] == 4) >= 12
+    assert sum(1 for c in SMALL if fused[c] == 7) >= 5
+    assert sum(1 for c in SMALL if special[c] == 7) >= 12
     assert fused[(2, 4, 32, 32, 8, 1, "f32", "f32")] == 1          # Q = 1: general ring kernel
-    assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 4
-    assert fused[(2, 16, 7, 7, 8, 2, "f32", "f32")] == 4
-    assert fused[(2, 3, 40, 24, 16, 2, "f32", "f32")] == 4
+    assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 7
+    assert fused[(2, 16, 7, 7, 8, 2, "f32", "f32")] == 7
+    assert fused[(2, 3, 40, 24, 16, 2, "f32", "f32")] == 7
     assert binding.div_plan_query(binding.make_desc(3, 4, 32, 32, 8, 2), NO_STRIP).fused == 1
     assert fused[(1, 2, 3, 3, 2, 2, "f32", "f32")] == 0          # sample is not a whole number of words
     assert fused[(2, 2, 70, 70, 64, 2, "f32", "f32")] == 0        # block wider than a warp
@@ -184,10 +186,10 @@ def test_fused_path_is_taken_where_expected():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
         nbytes = spec.numel * (4 if spec.x_dtype == "f32" else 2)
         first = 6 if (nbytes >= 56 * 2 ** 20 and spec.block == 8) else (3 if nbytes >= 20 * 2 ** 20 else 2)
-        assert binding.div_plan_query(d).fused == (first if spec.w % 4 == 0 else 4), spec.label()
-        assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 4), spec.label()
-        assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 4), spec.label()
-        assert binding.div_plan_query(d, STAGED).fused == (6 if spec.w % 4 == 0 else 4), spec.label()
+        assert binding.div_plan_query(d).fused == (first if spec.w % 4 == 0 else 7), spec.label()
+        assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 7), spec.label()
+        assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 7), spec.label()
+        assert binding.div_plan_query(d, STAGED).fused == (6 if spec.w % 4 == 0 else 7), spec.label()
         assert binding.div_plan_query(d).decompress_fast == (1 if spec.w % 4 == 0 else 2)
 
 
@@ -239,15 +241,17 @@ def test_same_seed_same_bytes_other_seed_other_codes():
     assert (wa != wc).mean() > 0.5
 
 
-@pytest.mark.parametrize("flags", [0, LAGGED, STAGED], ids=["strip_ring", "lagged", "staged"])
+@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL], ids=["strip_ring", "lagged", "staged", "planes_fused"])
 def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
     """Failure detection without a fault: the kernel waits for arrivals that never come, its 2 ms limit
     runs out, it records the timeout in the status word and returns; the context stays usable."""
     import ctypes
     spec = synth.config0()[0]
+    if flags == NO_SPECIAL:
+        spec = synth.TensorSpec(0, 0, 8, 64, 14, 14, "relu", "f32", "f32", 8, 2)      # a small-plane map
     x = to_device(synth.make_input(spec), "f32")
     codec = binding.Codec(*spec.shape, spec.block, spec.qbits)
-    assert codec.plan(flags).fused == {0: 2, LAGGED: 3, STAGED: 6}[flags]
+    assert codec.plan(flags).fused == {0: 2, LAGGED: 3, STAGED: 6, NO_SPECIAL: 7}[flags]
     st = binding.lib().div_debug_compress_starved(
         ctypes.byref(codec.desc), ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(codec.blob.data_ptr()), codec.blob.numel(),
         ctypes.c_void_p(codec.workspace.data_ptr()), codec.workspace.numel(), 0, ctypes.c_void_p(binding.current_stream_handle()),
@@ -269,7 +273,7 @@ def test_guard_bands_stay_untouched():
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
                  (2, 8, 32, 32, 8, 2, "bf16", "bf16")]:
         n, c, h, w, block, q, xd, ld = case
-        for flags in (0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
+        for flags in (0, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS):
             x = small_input(n, c, h, w, xd, seed=7)
             codec = binding.Codec(n, c, h, w, block, q, xd, ld)
             pad = 4096
@@ -377,6 +381,8 @@ def test_config2_other_paths_on_one_tensor():
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=LAGGED)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=RING)
     assert_sampled_parity(synth.config2()[2], 0, [0, 63], flags=STAGED)
+    assert_sampled_parity(synth.config2()[3], 0, [0, 63], flags=PLANES_PAIR)
+    assert_sampled_parity(synth.config2()[4], 0, [0, 63], flags=PLANES_PAIR)
     assert_sampled_parity(synth.config2()[0], 0, [17], flags=RING)
 
 
