@@ -35,16 +35,19 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM bytes per launch of profiled kernels come from profiles/traffic.json (written next to the ncu summaries):
 # each entry names the kernel, the map, dram__bytes_read.sum / dram__bytes_write.sum of one capture and the
-# SHA-256 of the kernel's source file at capture time.  An entry whose source has changed since is not used.
+# SHA-256 over the kernel's source files at capture time.  An entry whose sources have changed since is not used.
 def ncu_traffic(kernel: str, map_label: str):
     import hashlib
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
             table = json.load(f)
         e = table[f"{kernel} on {map_label}"]
-        with open(os.path.join(ROOT, e["source"]), "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest() != e["source_sha256"]:
-                return None
+        h = hashlib.sha256()
+        for rel in e["sources"]:
+            with open(os.path.join(ROOT, rel), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest() != e["sources_sha256"]:
+            return None
         return int(e["dram_bytes_read"]) + int(e["dram_bytes_write"])
     except Exception:
         return None

@@ -251,9 +251,12 @@ template <> struct StripRow2<__nv_bfloat16> {
 // rounding); returns the two results QUANT2_BITS + code.  Same integer as quant_bits(): with
 // F = 2^23 + field (the field dropped into the mantissa of 2^23), F * -2^-16 = -128 - u exactly, so one
 // fused multiply-add rounded towards +inf gives d = RU(t - u - 128), and ceil(d) = ceil(t - u) - 128
-// (rounding up never carries a value across an integer); the second add, rounded up onto the integer
-// grid of [2^23, 2^24), leaves that integer in the low mantissa bits.
-constexpr uint32_t QUANT2_BITS = MAGIC_CEIL_BITS - 128u;
+// (rounding up never carries a value across an integer); the second add, of 1.5 * 2^23 + 128 and rounded up
+// onto the integer grid of [2^23, 2^24), leaves ceil(t - u) in the low mantissa bits.  QUANT2_BITS has its
+// low 22 bits clear, so where the packed codes are stored as a byte or a half-word (Q = 2, 4) the bias of the
+// four results drops out of the stored bits by itself.
+constexpr uint32_t QUANT2_BITS = MAGIC_CEIL_BITS;
+constexpr float QUANT2_MAGIC = MAGIC_CEIL + 128.0f;
 __device__ __forceinline__ void quant2(uint64_t x01, uint64_t stored2, uint64_t delta2, uint64_t scale2, float qmax,
                                        uint32_t h, uint32_t& b0, uint32_t& b1) {
     const uint64_t t01 = mul2_rn(sub2_rn(sub2_rn(x01, stored2), delta2), scale2);
@@ -263,7 +266,7 @@ __device__ __forceinline__ void quant2(uint64_t x01, uint64_t stored2, uint64_t 
     t1 = fminf(t1, qmax);
     const uint64_t f01 = pk2u(__byte_perm(h, 0x4B000000u, 0x7610), __byte_perm(h, 0x4B000000u, 0x7632));   // 2^23 + field
     const uint64_t d01 = fma2_rp(f01, pk2(-1.52587890625e-05f, -1.52587890625e-05f), pk2(t0, t1));         // RU(t - u - 128)
-    upk2u(add2_rp(d01, pk2(MAGIC_CEIL, MAGIC_CEIL)), b0, b1);
+    upk2u(add2_rp(d01, pk2(QUANT2_MAGIC, QUANT2_MAGIC)), b0, b1);
 }
 
 // four elements of one strip row -> their codes packed Q bits apart (low bits first)
@@ -275,7 +278,9 @@ __device__ __forceinline__ uint32_t quant_row(uint64_t xy, uint64_t zw, uint64_t
     quant2(xy, stored2, delta2, scale2, qmax, (uint32_t)z, b0, b1);
     quant2(zw, stored2, delta2, scale2, qmax, (uint32_t)(z >> 32), b2, b3);
     constexpr uint32_t BIAS = QUANT2_BITS * (1u + (1u << Q) + (1u << (2 * Q)) + (1u << (3 * Q)));   // mod 2^32
-    return b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q)) - BIAS;
+    const uint32_t acc = b0 + (b1 << Q) + (b2 << (2 * Q)) + (b3 << (3 * Q));
+    if constexpr (4 * Q < 22) return acc;      // the caller stores the low 4 * Q bits only: the bias does not reach them
+    return acc - BIAS;
 }
 
 // the mixing function of the random stream (see rng_group) applied to a prepared counter
