@@ -368,7 +368,7 @@ def run_ours(args):
     build.build()
     binding.lib()
 
-    kernel_names_all = {7: "plane_fused_kernel", 6: "staged_kernel", 5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel",
+    kernel_names_all = {8: "line_fused_kernel", 7: "plane_fused_kernel", 6: "staged_kernel", 5: "line_stats_kernel + line_quant_kernel", 4: "plane_stats_kernel + plane_quant_kernel",
                         3: "lagged_kernel", 2: "fused_v_kernel", 1: "fused_compress_kernel", 0: "lfc_stats_kernel + quant_pack_kernel"}
     dec_names_all = {1: "decompress_quad_kernel", 2: "decompress_flat_kernel", 3: "decompress_line_kernel", 0: "decompress_general_kernel"}
     specs = synth.config_specs(2)

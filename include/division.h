@@ -104,8 +104,11 @@ typedef struct div_plan {
                                   planes (second read from L1 / L2); taken when all its CTAs can be resident;
                                4: the same in two launches;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;
-                               5: 1-D maps (h == 1; the appendix on 1D and 3D activation maps), W%4==0, B a power of two
-                                  in [4,128], Q in {2,4,8}: two launches, the second read comes from L2 */
+                               8: 1-D maps (h == 1; the appendix on 1D and 3D activation maps), W%4==0, B a power of two
+                                  in [4,128], Q in {2,4,8}, in one launch: a CTA owns a run of rows of one sample, joins
+                                  the sample's other CTAs through an arrival count and quantises the same rows (second
+                                  read from L1 / L2); taken when all its CTAs can be resident;
+                               5: the same in two launches */
     int32_t grid;           /* CTAs of the (first) compress kernel                            */
     int32_t threads;        /* threads per CTA                                                */
     int32_t stages;         /* shared-memory ring depth (ring kernels only)                   */
@@ -127,7 +130,7 @@ typedef struct div_plan {
 #define DIV_FLAG_NO_PLANE_KERNELS 8u /* never take the small-plane pair of kernels          */
 #define DIV_FLAG_NO_LINE_KERNELS 16u /* never take the pair of kernels for 1-D maps          */
 #define DIV_FLAG_NO_STAGED_KERNEL 32u/* never take the staged (bulk-copy rings) kernel       */
-#define DIV_FLAG_TWO_LAUNCH_PLANES 64u /* small planes: the pair of kernels, not the fused one */
+#define DIV_FLAG_TWO_LAUNCH_PLANES 64u /* small planes and 1-D maps: the pair of kernels, not the fused one */
 
 /*
  * Sizes of the cached tuple (H^L, V^H, Delta, delta) of Sec. 4.1 in the blob layout above:

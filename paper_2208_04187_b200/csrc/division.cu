@@ -178,6 +178,7 @@ struct Choice {
     VPlan vp;
     PlaneGeom pg;
     PlaneFusedPlan pf;
+    LineFused lf;
     FusedPlan fp;
 };
 
@@ -186,7 +187,7 @@ void choose_compress(const div_desc* d, const Shape& s, uint32_t flags, Choice* 
     c->code = 0;
     if (two_pass) return;
     if (!(flags & DIV_FLAG_NO_LINE_KERNELS) && plan_lines(d, s, &c->lg)) {
-        c->code = 5;
+        c->code = (!(flags & DIV_FLAG_TWO_LAUNCH_PLANES) && line_fused_applies(d, s, &c->lf)) ? 8 : 5;
         return;
     }
     const bool may_staged = !(flags & DIV_FLAG_NO_STAGED_KERNEL);
@@ -263,7 +264,12 @@ div_status div_plan_query(const div_desc* desc, uint32_t flags, div_plan* out) {
     Choice ch;
     choose_compress(desc, s, flags, &ch);
     out->fused = ch.code;
-    if (ch.code == 5) {
+    if (ch.code == 8) {
+        out->grid = (int32_t)(ch.lf.ctas_per_sample * s.N);
+        out->threads = 256;
+        out->chunk_elems = (int64_t)ch.lf.rpc * s.W;
+        out->chunks_per_sample = ch.lf.ctas_per_sample;
+    } else if (ch.code == 5) {
         out->grid = (int32_t)((ch.lg.qps + 256 * LINE_QPT - 1) / (256 * LINE_QPT) * s.N);
         out->threads = 256;
         out->chunk_elems = 4 * LINE_QPT * 256;
@@ -346,7 +352,8 @@ div_status div_compress_ex(const div_desc* desc, const void* x_dev, void* comp_d
         div_status r = DIV_OK;
         uint32_t drop = 0;
         switch (ch.code) {
-            case 5: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream);
+            case 8: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream, true);
+            case 5: return compress_lines(desc, s, lo, ch.lg, x_dev, blob, ws, seed, stream, false);
             case 6: r = compress_staged(desc, s, lo, ch.sp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STAGED_KERNEL; break;
             case 3: r = compress_lagged(desc, s, lo, ch.lp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_LAGGED_KERNEL; break;
             case 2: r = compress_fused_v(desc, s, lo, ch.vp, x_dev, blob, ws, seed, stream); drop = DIV_FLAG_NO_STRIP_KERNEL; break;

@@ -2,8 +2,10 @@
 // Minibatch x Channel x N, average pooling and nearest up-sampling along the last axis; Eq. 9 unchanged).
 // A 1-D map is described as N x C x 1 x W.  Conditions: W % 4 == 0, B a power of two in [4, 128], Q in {2, 4, 8}.
 //
-// Two launches, no dependency inside a kernel (token / MLP activations of one layer are tens of MB: the second
-// read of x comes from the 126 MB L2; larger tensors are still handled correctly, reading x twice from HBM):
+// line_fused_kernel does both halves in one launch (see there); where its CTAs cannot all be resident the pair
+// below runs instead.  Two launches, no dependency inside a kernel (token / MLP activations of one layer are tens
+// of MB: the second read of x comes from the 126 MB L2; larger tensors are still handled correctly, reading x
+// twice from HBM):
 //   line_stats_kernel   a lane owns 4 consecutive elements; the B/4 lanes of a block meet through xor shuffles
 //                       (the balanced pairwise tree over the B positions, neighbours first); stored
 //                       low-frequency values; residual extremes -> per-sample min / max keys in the scratch slots
@@ -120,6 +122,154 @@ line_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const ui
     }
 }
 
+// One launch for both halves.  CTA (b, n) owns the rows [b * rpc, (b + 1) * rpc) of sample n:
+//   1. block means, stored low-frequency values and residual extremes of its rows, exactly as line_stats_kernel;
+//      the CTA's extremes are folded into the sample's slot (two reductions without an answer), then, behind a
+//      release fence, the CTA is counted as arrived;
+//   2. thread 0 waits (bounded) until all CTAs of the sample have arrived and derives (delta, Delta, scale);
+//   3. Eq. 9 and packing of the same rows as line_quant_kernel: x is read a second time (it is still in this
+//      SM's L1 or in the L2), the low-frequency values are the ones this CTA stored in step 1.
+// The launch is cooperative so that the CTAs a wait depends on are resident; no grid-wide barrier is used.
+struct LineFused {
+    uint32_t rpc;                 // rows per CTA
+    uint32_t ctas_per_sample;
+    uint32_t expected;            // arrivals that complete a sample
+    uint64_t timeout_ns;
+};
+
+template <typename XT, typename LT, int Q>
+__global__ void __launch_bounds__(256)
+line_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, void* __restrict__ packed_v,
+                  float* __restrict__ stats, LineGeom g, LineFused f, uint64_t seed) {
+    typedef typename PackedUnit<Q>::type OutT;
+    __shared__ uint32_t s_kmin, s_kmax, s_delta, s_scale, s_ok;
+    const uint32_t n = blockIdx.y;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t lpt = 1u << g.log2lpt;
+    const uint32_t row0 = blockIdx.x * f.rpc;
+    const uint32_t nrows = row0 < g.C ? min(f.rpc, g.C - row0) : 0u;
+    const XT* x_n = x + (size_t)n * g.CHW;
+    LT* lfc_n = lfc + (size_t)n * g.C * g.Wb;
+    if (threadIdx.x == 0) {
+        s_kmin = 0;
+        s_kmax = 0;
+        s_ok = 0;
+    }
+    __syncthreads();
+
+    // ---------------- half 1: a lane owns 4 consecutive elements; warp chunks of this CTA's rows ----------------
+    {
+        const uint32_t c0 = row0 * g.cpr, c1 = (row0 + nrows) * g.cpr;       // this CTA's warp chunks [c0, c1)
+        float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+        for (uint32_t wc0 = c0 + warp * LINE_U; wc0 < c1; wc0 += 8u * LINE_U) {
+            uint64_t xy[LINE_U], zw[LINE_U];
+            uint32_t row[LINE_U], q[LINE_U];
+            bool ok[LINE_U];
+#pragma unroll
+            for (int u = 0; u < LINE_U; ++u) {
+                const uint32_t wc = wc0 + u;
+                const bool live = wc < c1;
+                row[u] = fdiv(live ? wc : c0, g.by_cpr);
+                q[u] = ((live ? wc : c0) - row[u] * g.cpr) * 32u + lane;          // quad inside the row
+                ok[u] = live && q[u] < g.qpr;
+                xy[u] = 0ull;
+                zw[u] = 0ull;
+                if (ok[u]) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (row[u] * g.W + 4u * q[u])), xy[u], zw[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < LINE_U; ++u) {
+                float a, b, c, d;
+                upk2(xy[u], a, b);
+                upk2(zw[u], c, d);
+                float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
+                for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+                const uint32_t t = q[u] >> g.log2lpt;                         // block inside the row
+                const bool tail = t + 1u == g.Wb;
+                const float inv = tail ? g.inv_tail : g.inv_full;
+                const float mean = (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, tail ? g.cnt_tail : g.cnt_full);
+                const float stored = Elem<LT>::round(mean);
+                if (ok[u]) {
+                    if ((q[u] & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (row[u] * g.Wb + t), mean);
+                    lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
+                    hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
+                }
+            }
+        }
+        const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
+        const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
+        if (lane == 0) {
+            atomicMax(&s_kmin, kmin);
+            atomicMax(&s_kmax, kmax);
+        }
+    }
+    // the barrier also orders this CTA's stores of low-frequency values before its loads of them in half 2
+    __syncthreads();
+
+    // ---------------- the sample's extremes: fold, count, wait for the other CTAs of the sample ----------------
+    if (threadIdx.x == 0) {
+        uint32_t* slot = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+        if (nrows) {
+            red_max_relaxed(slot + 0, s_kmin);
+            red_max_relaxed(slot + 1, s_kmax);
+        }
+        fence_acq_rel_gpu();
+        asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(slot + 2), "r"(1u) : "memory");
+        uint32_t polls = 0;
+        uint64_t t0 = 0;
+        bool ok = true;
+        while (ld_acquire_u32(slot + 2) != f.expected) {
+            if ((++polls & 7u) == 0) {
+                const uint64_t tn = now_ns();
+                if (t0 == 0) t0 = tn;
+                if (ld_relaxed_u32(ws) != 0u || tn - t0 > f.timeout_ns) {
+                    atomicCAS(ws, 0u, (uint32_t)DIV_ERR_TIMEOUT);
+                    atomicCAS(ws + 1, 0u, n + 1u);
+                    ok = false;
+                    break;
+                }
+            }
+            __nanosleep(100);
+        }
+        if (ok) {
+            const QParams qp = make_qparams(key_float(~ld_relaxed_u32(slot + 0)), key_float(ld_relaxed_u32(slot + 1)), Q);
+            if (blockIdx.x == 0) {
+                stats[2 * (size_t)n + 0] = qp.delta;
+                stats[2 * (size_t)n + 1] = qp.step;
+            }
+            s_delta = __float_as_uint(qp.delta);
+            s_scale = __float_as_uint(qp.scale);
+            s_ok = 1;
+        }
+    }
+    __syncthreads();
+    if (!s_ok || nrows == 0) return;
+
+    // ---------------- half 2: a thread per 4 consecutive elements of the CTA's rows ----------------
+    const float delta = __uint_as_float(s_delta), scale = __uint_as_float(s_scale);
+    const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
+    const uint64_t base = rng_sample_base(seed, n);
+    OutT* packed = reinterpret_cast<OutT*>(packed_v) + (uint64_t)n * g.qps;
+    const uint32_t qa = row0 * g.qpr, qb = (row0 + nrows) * g.qpr;           // this CTA's quads [qa, qb)
+    for (uint32_t q0 = qa + threadIdx.x; q0 < qb; q0 += 256u * 4u) {
+        uint64_t xy[4], zw[4];
+        float lf[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t q = q0 + k * 256u;
+            if (q < qb) {
+                StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + q * 4u), xy[k], zw[k]);
+                const uint32_t row = fdiv(q, g.by_qpr);
+                lf[k] = Elem<LT>::load_cg(lfc_n + (row * g.Wb + ((q - row * g.qpr) >> g.log2lpt)));      // stored by other warps of this CTA
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t q = q0 + k * 256u;
+            if (q < qb) packed[q] = (OutT)quant_row<Q>(xy[k], zw[k], pk2(lf[k], lf[k]), delta2, scale2, rng_group(base, q));
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -151,11 +301,80 @@ inline bool plan_lines(const div_desc* d, const Shape& s, LineGeom* out) {
     return true;
 }
 
+template <typename XT, typename LT, int Q>
+inline int line_fused_occupancy(int dev) {
+    static SmemSeen cached[DEVICE_CACHE_SLOTS];          // .bytes holds the count
+    const void* kern = (const void*)line_fused_kernel<XT, LT, Q>;
+    const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
+    if (slot && cached[dev].fn.load(std::memory_order_acquire) == kern) {
+        const int c = cached[dev].bytes.load(std::memory_order_acquire);
+        if (c > 0) return c;
+    }
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, line_fused_kernel<XT, LT, Q>, 256, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    if (slot && n > 0) {
+        cached[dev].fn.store(nullptr, std::memory_order_release);
+        cached[dev].bytes.store(n, std::memory_order_release);
+        cached[dev].fn.store(kern, std::memory_order_release);
+    }
+    return n;
+}
+
+// rows per CTA and CTAs per sample of the single-launch form; false when its CTAs could not all be resident
+template <typename XT, typename LT, int Q>
+inline bool plan_line_fused(const Shape& s, const DeviceInfo& di, LineFused* out) {
+    const int occ = line_fused_occupancy<XT, LT, Q>(di.dev);
+    if (occ < 1) return false;
+    const uint64_t capacity = (uint64_t)occ * di.sms;
+    if (s.N > capacity) return false;
+    uint64_t want = (8ull * di.sms + s.N - 1) / s.N;                     // CTAs per sample: about 8 per SM in all ...
+    if (want * s.N > capacity) want = capacity / s.N;                    // ... and never more than fit at once
+    if (want > s.C) want = s.C;
+    if (want < 1) want = 1;
+    out->rpc = (uint32_t)((s.C + want - 1) / want);
+    out->ctas_per_sample = (s.C + out->rpc - 1) / out->rpc;
+    out->expected = out->ctas_per_sample;
+    out->timeout_ns = 2000000000ull;
+    return true;
+}
+
+template <typename XT, typename LT, int Q>
+inline bool launch_line_fused(const Shape& s, const div_layout& lo, const LineGeom& g, const DeviceInfo& di, const void* x,
+                              uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+    LineFused f;
+    if (!plan_line_fused<XT, LT, Q>(s, di, &f)) return false;
+    const XT* xt = (const XT*)x;
+    LT* lfc = (LT*)(blob + lo.lfc_off);
+    void* packed = blob + lo.packed_off;
+    float* stats = (float*)(blob + lo.stats_off);
+    LineGeom gg = g;
+    void* args[] = {(void*)&xt, (void*)&lfc, (void*)&ws, (void*)&packed, (void*)&stats, (void*)&gg, (void*)&f, (void*)&seed};
+    if (cudaLaunchCooperativeKernel((const void*)line_fused_kernel<XT, LT, Q>, dim3(f.ctas_per_sample, s.N), dim3(256), args, 0, st) !=
+        cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
 template <typename XT, typename LT>
 inline div_status compress_lines_t(const div_desc* d, const Shape& s, const div_layout& lo, const LineGeom& g,
-                                   const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+                                   const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, bool allow_fused) {
     const DeviceInfo di = device_info();
     if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
+    if (allow_fused) {
+        bool done = false;
+        switch (d->qbits) {
+            case 2: done = launch_line_fused<XT, LT, 2>(s, lo, g, di, x, blob, ws, seed, st); break;
+            case 4: done = launch_line_fused<XT, LT, 4>(s, lo, g, di, x, blob, ws, seed, st); break;
+            case 8: done = launch_line_fused<XT, LT, 8>(s, lo, g, di, x, blob, ws, seed, st); break;
+            default: return DIV_ERR_PARAM;
+        }
+        if (done) return DIV_OK;
+    }
     // pass 1: enough CTAs per sample to fill the GPU a few times over, never more than there are warp chunks
     uint32_t bx = (uint32_t)((16ull * di.sms + s.N - 1) / s.N);
     const uint32_t bx_max = (g.chunks + 8u * LINE_U - 1u) / (8u * LINE_U);
@@ -179,14 +398,25 @@ inline div_status compress_lines_t(const div_desc* d, const Shape& s, const div_
 }
 
 inline div_status compress_lines(const div_desc* d, const Shape& s, const div_layout& lo, const LineGeom& g,
-                                 const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
+                                 const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, bool allow_fused = true) {
     typedef __nv_bfloat16 bf16;
     if (d->x_dtype == DIV_F32) {
-        if (d->lfc_dtype == DIV_F32) return compress_lines_t<float, float>(d, s, lo, g, x, blob, ws, seed, st);
-        return compress_lines_t<float, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+        if (d->lfc_dtype == DIV_F32) return compress_lines_t<float, float>(d, s, lo, g, x, blob, ws, seed, st, allow_fused);
+        return compress_lines_t<float, bf16>(d, s, lo, g, x, blob, ws, seed, st, allow_fused);
     }
-    if (d->lfc_dtype == DIV_F32) return compress_lines_t<bf16, float>(d, s, lo, g, x, blob, ws, seed, st);
-    return compress_lines_t<bf16, bf16>(d, s, lo, g, x, blob, ws, seed, st);
+    if (d->lfc_dtype == DIV_F32) return compress_lines_t<bf16, float>(d, s, lo, g, x, blob, ws, seed, st, allow_fused);
+    return compress_lines_t<bf16, bf16>(d, s, lo, g, x, blob, ws, seed, st, allow_fused);
+}
+
+// would the single-launch form run this descriptor?
+inline bool line_fused_applies(const div_desc* d, const Shape& s, LineFused* out) {
+    typedef __nv_bfloat16 bf16;
+    const DeviceInfo di = device_info();
+    if (!di.ok || di.sms < 1) return false;
+#define DIVK_LQ(XT, LT) (d->qbits == 2 ? plan_line_fused<XT, LT, 2>(s, di, out) : d->qbits == 4 ? plan_line_fused<XT, LT, 4>(s, di, out) : plan_line_fused<XT, LT, 8>(s, di, out))
+    if (d->x_dtype == DIV_F32) return d->lfc_dtype == DIV_F32 ? DIVK_LQ(float, float) : DIVK_LQ(float, bf16);
+    return d->lfc_dtype == DIV_F32 ? DIVK_LQ(bf16, float) : DIVK_LQ(bf16, bf16);
+#undef DIVK_LQ
 }
 
 }  // namespace divk
