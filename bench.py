@@ -706,7 +706,7 @@ def run_ours(args):
 
     # ---- the other workload configurations, tensor by tensor ----
     other_configs = None
-    if args.configs and not args.maps:
+    if args.configs and not args.maps and rank == 0:
         dev_x.clear()                   # hand the benchmark's device buffers back first
         dev_out.clear()
         for c in codecs:

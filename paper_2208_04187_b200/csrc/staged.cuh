@@ -54,6 +54,9 @@ namespace divk {
 #ifndef DIVK_S_AHEAD
 #define DIVK_S_AHEAD 4
 #endif
+#ifndef DIVK_S_Q_STAGES_PER_8
+#define DIVK_S_Q_STAGES_PER_8 4
+#endif
 #ifndef DIVK_S_REDUCE_WARPS
 #define DIVK_S_REDUCE_WARPS 14
 #endif
@@ -77,6 +80,7 @@ struct SPlan {
     uint32_t kr, kq;               // stages of the reduce ring / of the quantise ring
     uint32_t G;                    // bands per full chunk
     uint32_t spb;                  // strip slots per band
+    uint32_t paired;               // 1: bands are laid out in pairs, their single-strip last tiles side by side (see the table)
     uint32_t slots;                // G * spb strip slots per full chunk
     uint32_t nf;                   // units per full chunk
     uint32_t chunk_elems;          // elements of a full chunk
@@ -108,7 +112,7 @@ struct SParams {
 
 // what a producer posts beside a stage before it issues the copy
 struct SDesc {
-    uint32_t nslots;               // strip slots of the chunk
+    uint32_t ntiles;               // tiles of the chunk (a short last chunk of a sample has fewer)
     uint32_t n;                    // sample
     uint32_t tile0;                // first tile of the chunk inside the sample
     uint32_t seq;                  // 1 + index (in this CTA's list) of the chunk the stage holds; written last (see s_wait_chunk)
@@ -211,18 +215,19 @@ __device__ __forceinline__ bool s_wait_chunk(uint64_t* bar, uint32_t parity, con
 // the B rows of a strip from a stage; rows at or past `rows` read as zero (full: every lane has all B rows)
 template <typename XT, int P2>
 __device__ __forceinline__ void s_load_strip(const unsigned char* xs, uint32_t row_bytes, uint32_t rows, bool full,
-                                             uint64_t (&vxy)[P2], uint64_t (&vzw)[P2]) {
+                                             uint32_t rmax, uint64_t (&vxy)[P2], uint64_t (&vzw)[P2]) {
     if (full) {
 #pragma unroll
         for (int r = 0; r < P2; ++r) StripRow2<XT>::load(xs + r * row_bytes, vxy[r], vzw[r]);
     } else {
 #pragma unroll
         for (int r = 0; r < P2; ++r) {
-            if ((uint32_t)r < rows) {
-                StripRow2<XT>::load(xs + r * row_bytes, vxy[r], vzw[r]);
-            } else {
-                vxy[r] = 0ull;
-                vzw[r] = 0ull;
+            vxy[r] = 0ull;
+            vzw[r] = 0ull;
+            // rmax, the largest row count in the warp, is the same in every lane: a unit of short bands only
+            // steps over its missing rows without issuing anything for them
+            if ((uint32_t)r < rmax) {
+                if ((uint32_t)r < rows) StripRow2<XT>::load(xs + r * row_bytes, vxy[r], vzw[r]);
             }
         }
     }
@@ -231,8 +236,8 @@ __device__ __forceinline__ void s_load_strip(const unsigned char* xs, uint32_t r
 // tile mean in the fixed order (balanced tree down the rows of each of the 4 columns, then across the
 // columns of the strip, then across the strips of the tile); every lane of the warp must call it
 template <int P2>
-__device__ __forceinline__ float s_tile_mean(const uint64_t (&vxy)[P2], const uint64_t (&vzw)[P2], bool active, float inv,
-                                             float cnt) {
+__device__ __forceinline__ float s_tile_mean(const uint64_t (&vxy)[P2], const uint64_t (&vzw)[P2], bool active, bool mate,
+                                             float inv, float cnt) {
     constexpr uint32_t LPT = P2 / 4;
     uint64_t cxy[P2 / 2], czw[P2 / 2];
 #pragma unroll
@@ -253,8 +258,11 @@ __device__ __forceinline__ float s_tile_mean(const uint64_t (&vxy)[P2], const ui
     upk2(czw[0], c2, c3);
     float sum = __fadd_rn(__fadd_rn(c0, c1), __fadd_rn(c2, c3));
     if (!active) sum = 0.f;                                 // a padding lane stands for columns past the right edge
-#pragma unroll
-    for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+    if (LPT == 2u) {
+        // the tile's other strip is next door; a tile of one strip adds the zero its missing columns stand for
+        const float other = __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+        sum = __fadd_rn(sum, mate ? other : 0.f);
+    }
     return (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, cnt);
 }
 
@@ -283,25 +291,57 @@ staged_kernel(const SParams p) {
     const uint32_t n_my = blockIdx.x < TU ? (TU - blockIdx.x + G - 1u) / G : 0u;
 
     // ---- set-up: strip table, barriers ----
+    // One entry per strip slot of a full chunk; slot sl is lane sl % 32 of unit sl / 32.
     //   bits 0-12 offset of the strip's first element inside the chunk, in groups of 4 elements; 13-16 in-bounds rows
-    //   (0: padding slot); 17-18 kind of tile; 19 writes the tile's mean; 20-31 tile inside the chunk
-    for (uint32_t sl = threadIdx.x; sl < p.pl.slots; sl += blockDim.x) {
-        const uint32_t band = sl / p.pl.spb, q = sl - band * p.pl.spb;
-        const uint32_t col0 = 4u * q;
-        const bool ok = col0 < s.W;
-        uint32_t eoff, rows;
-        if (p.pl.uniform) {
-            eoff = band * s.B * s.W + col0;
-            rows = s.B;
-        } else {
-            const uint32_t pl_ = band / s.Hb, bh = band - pl_ * s.Hb;
-            eoff = pl_ * s.HW + bh * s.B * s.W + col0;
-            rows = (bh + 1u == s.Hb) ? p.tail_rows : s.B;
+    //   (0: padding slot); 17-18 kind of tile; 19 writes the tile's mean (first strip of its tile); 20 the tile has a
+    //   second strip, held by the lane next door (lane ^ 1); 21-31 tile inside the chunk.
+    // Order of the slots: bands of full height first, then the short last bands of the planes, so that most units
+    // hold strips of one height only.  Inside a band the strips follow each other, 2 per tile for B = 8.  Where W / 4
+    // is odd the last tile of a band has one strip; bands are then laid out in pairs, their two-strip tiles first and
+    // the two single strips side by side, so that every two-strip tile starts on an even lane and no lane is idle.
+    {
+        const uint32_t spr = s.W >> 2;                                       // strips per band that exist
+        const uint32_t full_bands = p.pl.uniform ? p.pl.G : (p.pl.G / s.Hb) * (s.Hb - 1u);
+        for (uint32_t sl = threadIdx.x; sl < p.pl.slots; sl += blockDim.x) {
+            uint32_t ob, q;                                                  // band in the order above, strip inside the band
+            if (p.pl.paired) {
+                const uint32_t pair = sl / (2u * spr), r = sl - pair * 2u * spr;
+                const uint32_t two = 2u * (spr - 1u);                        // lanes of the pair's two-strip tiles
+                if (r < two) {
+                    const uint32_t t = r >> 1, per = (spr - 1u) >> 1;        // two-strip tiles per band
+                    const uint32_t wb = t / per;
+                    ob = 2u * pair + wb;
+                    q = 2u * (t - wb * per) + (r & 1u);
+                } else {
+                    ob = 2u * pair + (r - two);
+                    q = spr - 1u;
+                }
+            } else {
+                ob = sl / p.pl.spb;
+                q = sl - ob * p.pl.spb;
+            }
+            uint32_t band;                                                   // band inside the chunk, in memory order
+            if (p.pl.uniform) band = ob;
+            else if (ob < full_bands) band = ob + ob / (s.Hb - 1u);
+            else band = (ob - full_bands) * s.Hb + (s.Hb - 1u);
+            const uint32_t col0 = 4u * q;
+            const bool ok = col0 < s.W;
+            uint32_t eoff, rows;
+            if (p.pl.uniform) {
+                eoff = band * s.B * s.W + col0;
+                rows = s.B;
+            } else {
+                const uint32_t pl_ = band / s.Hb, bh = band - pl_ * s.Hb;
+                eoff = pl_ * s.HW + bh * s.B * s.W + col0;
+                rows = (bh + 1u == s.Hb) ? p.tail_rows : s.B;
+            }
+            const uint32_t bw = q / LPT;
+            const uint32_t which = ((rows != s.B) ? 2u : 0u) + ((bw == s.Wb - 1u && (s.W % s.B) != 0u) ? 1u : 0u);
+            const uint32_t writer = (q % LPT) == 0 ? 1u : 0u;
+            const uint32_t mate = (LPT == 2u && !(p.pl.paired && q == spr - 1u)) ? 1u : 0u;
+            table[sl] = (ok ? (eoff >> 2) : 0u) | ((ok ? rows : 0u) << 13) | (which << 17) | (writer << 19) | (mate << 20) |
+                        ((band * s.Wb + bw) << 21);
         }
-        const uint32_t bw = q / LPT;
-        const uint32_t which = ((rows != s.B) ? 2u : 0u) + ((bw == s.Wb - 1u && (s.W % s.B) != 0u) ? 1u : 0u);
-        const uint32_t writer = (q % LPT) == 0 ? 1u : 0u;
-        table[sl] = (ok ? (eoff >> 2) : 0u) | ((ok ? rows : 0u) << 13) | (which << 17) | (writer << 19) | ((band * s.Wb + bw) << 20);
     }
     if (threadIdx.x == 0) {
         for (uint32_t i = 0; i < (uint32_t)S_MAX_STAGES; ++i) {
@@ -449,7 +489,7 @@ staged_kernel(const SParams p) {
             const uint32_t nelem = min(p.pl.chunk_elems, s.CHW - e0);
             const uint32_t nbands = min(p.pl.G, p.pl.bands_per_sample - k * p.pl.G);
             SDesc d;
-            d.nslots = nbands * p.pl.spb;
+            d.ntiles = nbands * s.Wb;
             d.n = n;
             d.tile0 = k * p.pl.G * s.Wb;
             d.seq = 0;
@@ -502,32 +542,38 @@ staged_kernel(const SParams p) {
             if (!landed) break;
             // every unit index takes part in the closing count, also where a short chunk has no strips for it:
             // a stage is recycled only after each of its nf readers has looked at it
-            const uint32_t nslots = ctl->desc_r[st].nslots;
-            const bool work = k * 32u < nslots;
+            // (a short last chunk of a sample holds a prefix of the tiles in memory order, not of the table: its
+            // lanes are masked one by one)
+            const uint32_t ntiles = ctl->desc_r[st].ntiles;
+            uint32_t rec = 0u;
+            {
+                const uint32_t sl = k * 32u + lane;
+                if (sl < p.pl.slots) rec = table[sl];
+                if ((rec >> 21) >= ntiles) rec = 0u;
+            }
+            const bool work = __any_sync(0xFFFFFFFFu, rec != 0u);
             uint32_t kmin = 0, kmax = 0;
             if (work) {
                 const uint32_t n = ctl->desc_r[st].n;
-                const uint32_t sl = k * 32u + lane;
-                uint32_t rec = 0u;
-                if (sl < nslots) rec = table[sl];
                 const uint32_t rows = (rec >> 13) & 15u;
                 const bool active = rows != 0u;
                 const uint32_t which = (rec >> 17) & 3u;
                 const unsigned char* xs = ring_r + (size_t)st * stage_bytes + ((size_t)(rec & 0x1FFFu) << QSHIFT);
                 const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
                 uint64_t vxy[P2], vzw[P2];
-                s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
-                const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
+                const uint32_t rmax = full ? (uint32_t)P2 : __reduce_max_sync(0xFFFFFFFFu, rows);
+                s_load_strip<XT, P2>(xs, row_bytes, rows, full, rmax, vxy, vzw);
+                const float mean = s_tile_mean<P2>(vxy, vzw, active, (rec >> 20) & 1u, p.inv_cnt[which], p.cnt[which]);
                 const float stored = Elem<LT>::round(mean);
                 float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
                 if (active) {
                     if (rec & (1u << 19))
-                        Elem<LT>::store(lfc_out + (size_t)n * s.C * s.TPP + ctl->desc_r[st].tile0 + (rec >> 20), mean);
+                        Elem<LT>::store(lfc_out + (size_t)n * s.C * s.TPP + ctl->desc_r[st].tile0 + (rec >> 21), mean);
                     // extremes of x over the strip's in-bounds rows; x -> fl(x - stored) is monotone
                     float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
 #pragma unroll
                     for (int r = 0; r < P2; ++r) {
-                        if (full || (uint32_t)r < rows) {
+                        if (full || ((uint32_t)r < rmax && (uint32_t)r < rows)) {
                             float a_, b_, c_, d_;
                             upk2(vxy[r], a_, b_);
                             upk2(vzw[r], c_, d_);
@@ -598,11 +644,14 @@ staged_kernel(const SParams p) {
         const uint32_t round = fdiv(it, p.by_kq);
         const uint32_t st = it - round * KQ;
         if (!__all_sync(0xFFFFFFFFu, s_wait_chunk(&ctl->full_q[st], round & 1u, &ctl->desc_q[st].seq, it, p, ctl))) break;
-        const uint32_t nslots = ctl->desc_q[st].nslots;
-        if (k * 32u < nslots) {
+        const uint32_t ntiles = ctl->desc_q[st].ntiles;
+        uint32_t rec = 0u;
+        {
             const uint32_t sl = k * 32u + lane;
-            uint32_t rec = 0u;
-            if (sl < nslots) rec = table[sl];
+            if (sl < p.pl.slots) rec = table[sl];
+            if ((rec >> 21) >= ntiles) rec = 0u;
+        }
+        if (__any_sync(0xFFFFFFFFu, rec != 0u)) {
             const uint32_t rows = (rec >> 13) & 15u;
             const bool active = rows != 0u;
             const uint32_t which = (rec >> 17) & 3u;
@@ -610,8 +659,9 @@ staged_kernel(const SParams p) {
             const unsigned char* xs = ring_q + (size_t)st * stage_bytes + ((size_t)quad << QSHIFT);
             const bool full = __all_sync(0xFFFFFFFFu, rows == (uint32_t)P2 || rows == 0u);
             uint64_t vxy[P2], vzw[P2];
-            s_load_strip<XT, P2>(xs, row_bytes, rows, full, vxy, vzw);
-            const float mean = s_tile_mean<P2>(vxy, vzw, active, p.inv_cnt[which], p.cnt[which]);
+            const uint32_t rmax = full ? (uint32_t)P2 : __reduce_max_sync(0xFFFFFFFFu, rows);
+            s_load_strip<XT, P2>(xs, row_bytes, rows, full, rmax, vxy, vzw);
+            const float mean = s_tile_mean<P2>(vxy, vzw, active, (rec >> 20) & 1u, p.inv_cnt[which], p.cnt[which]);
             const float stored = Elem<LT>::round(mean);
             if (active) {
                 const float delta = ctl->desc_q[st].delta, scale = ctl->desc_q[st].scale;
@@ -629,10 +679,12 @@ staged_kernel(const SParams p) {
                 } else {
 #pragma unroll
                     for (int r = 0; r < P2; ++r) {
-                        if ((uint32_t)r < rows) {
-                            *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
-                            out += W4;
-                            ctr += p.rng_row_step;
+                        if ((uint32_t)r < rmax) {
+                            if ((uint32_t)r < rows) {
+                                *out = (OutT)quant_row<Q>(vxy[r], vzw[r], stored2, delta2, scale2, rng_mix(ctr));
+                                out += W4;
+                                ctr += p.rng_row_step;
+                            }
                         }
                     }
                 }
@@ -672,15 +724,18 @@ inline div_status plan_staged(const div_desc* d, const Shape& s, SPlan* out) {
     if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
 
     SPlan pl = SPlan();
-    pl.spb = s.Wb * (s.P2 / 4);
+    pl.spb = s.W / 4u;
+    pl.paired = (s.P2 == 8u && (pl.spb & 1u)) ? 1u : 0u;
     const uint64_t bands = (uint64_t)s.C * s.Hb;
     if (bands >= (1ull << 31)) return DIV_ERR_PARAM;
     pl.bands_per_sample = (uint32_t)bands;
     pl.uniform = (s.H % s.B == 0) ? 1u : 0u;
     // bands per chunk: a count that keeps the chunk's inner geometry the same for every chunk (any count when
     // all bands are alike, whole planes otherwise) and, where possible, fills whole units of 32 strips
-    const uint32_t geo = pl.uniform ? 1u : s.Hb;
-    const uint64_t geo_bytes = pl.uniform ? (uint64_t)s.B * s.W * sx : (uint64_t)s.HW * sx;     // bytes of `geo` bands
+    // (an even count where the table lays bands out in pairs)
+    const uint32_t geo1 = pl.uniform ? 1u : s.Hb;
+    const uint32_t geo = (pl.paired && (geo1 & 1u)) ? 2u * geo1 : geo1;
+    const uint64_t geo_bytes = (pl.uniform ? (uint64_t)s.B * s.W * sx : (uint64_t)s.HW * sx) * (geo / geo1);     // bytes of `geo` bands
     const uint32_t fill = 32u / gcd_u32(32u, pl.spb);
     const uint32_t both = lcm_u32(geo, fill);
     const uint64_t both_bytes = geo_bytes * (both / geo);
@@ -693,19 +748,24 @@ inline div_status plan_staged(const div_desc* d, const Shape& s, SPlan* out) {
     if (G > bands_up) G = bands_up;
     pl.G = G;
     pl.slots = G * pl.spb;
-    if (pl.slots > 4096u || G * s.Wb > 4096u) return DIV_ERR_PARAM;         // widths of the strip table's fields
+    if (pl.slots > 4096u || G * s.Wb > 2048u) return DIV_ERR_PARAM;         // widths of the strip table's fields
     pl.nf = (pl.slots + 31u) / 32u;
     pl.chunk_elems = pl.uniform ? G * s.B * s.W : (G / s.Hb) * s.HW;
     if (pl.chunk_elems >= (1u << 15)) return DIV_ERR_PARAM;
     pl.chunks_per_sample = (pl.bands_per_sample + G - 1u) / G;
     pl.stage_bytes = (pl.chunk_elems * sx + 127u) & ~127u;
-    // shared memory: the two rings, the strip table, the control block; as many stages as fit, half of them
-    // (rounded down) for the quantise ring, whose copies come from the L2 and land sooner
+    // shared memory: the two rings, the strip table, the control block; as many stages as fit, DIVK_S_Q_STAGES_PER_8
+    // eighths of them (rounded down) for the quantise ring
     const uint32_t fixed = ((pl.slots * 4u + 15u) & ~15u) + (uint32_t)sizeof(SCtl) + 16u;
     if ((uint32_t)di.smem_optin < fixed + 4u * pl.stage_bytes) return DIV_ERR_PARAM;
     uint32_t stages = ((uint32_t)di.smem_optin - fixed) / pl.stage_bytes;
     if (stages > 2u * S_MAX_STAGES) stages = 2u * S_MAX_STAGES;
-    const uint32_t kq = stages / 2u, kr = stages - kq;
+    uint32_t kq = stages * DIVK_S_Q_STAGES_PER_8 / 8u;
+    if (kq < 2u) kq = 2u;
+    if (kq > stages - 2u) kq = stages - 2u;
+    if (kq > (uint32_t)S_MAX_STAGES) kq = S_MAX_STAGES;
+    uint32_t kr = stages - kq;
+    if (kr > (uint32_t)S_MAX_STAGES) kr = S_MAX_STAGES;
     pl.kr = kr;
     pl.kq = kq;
     pl.smem_bytes = (int32_t)((kr + kq) * pl.stage_bytes + fixed);
