@@ -225,9 +225,11 @@ decompress_line_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
 // ---------------------------------------------------------------------------------------------
 // flat kernel: any W and B, sample size a multiple of 4 elements, planes of at most FLAT_MAX_HW
 // elements.  One thread produces QPT quads of 4 consecutive elements (global flat order), which may
-// lie in different tiles, rows or planes: the tile of every position of a plane comes from a table
-// in shared memory (built once per CTA), the plane index advances with the position; the low-frequency
-// values of the planes a CTA touches are staged in shared memory too.
+// lie in different tiles, rows or planes.  Where the 4 low-frequency values of a quad sit repeats every
+// lcm(HW, 4) elements, so a table in shared memory (built once per CTA) holds, for every quad of one such
+// period, the 4 offsets (plane inside the period * tiles per plane + tile inside the plane) as 16-bit numbers:
+// one 8-byte load per quad instead of a walk over positions.  The low-frequency values of the planes a CTA
+// touches are staged in shared memory too.
 // grid = (ceil(quads_per_sample / (256*QPT)), N), dynamic shared memory = flat_smem_bytes()
 // ---------------------------------------------------------------------------------------------
 constexpr uint32_t FLAT_MAX_HW = 8192;
@@ -235,15 +237,36 @@ constexpr uint32_t FLAT_MAX_HW = 8192;
 struct DecFlat {
     uint32_t qps;        // quads per sample = CHW / 4
     uint32_t C, TPP, Wb, HW, W, B;
-    uint32_t table_words;    // 32-bit words the tile table takes in shared memory
+    uint32_t table_words;    // 32-bit words the quad table takes in shared memory
     uint32_t planes_per_cta; // upper bound of the planes one CTA touches
-    FastDiv by_hw, by_w, by_b;
+    uint32_t period;         // quads after which the quad table repeats
+    uint32_t period_planes;  // planes one period covers (1, 2 or 4)
+    FastDiv by_hw, by_w, by_b, by_period;
 };
 // planes a run of `elems` consecutive elements can touch, and the dynamic shared memory of the flat kernels
 inline uint32_t flat_planes_per_cta(uint32_t elems, uint32_t hw) { return (elems + hw - 1) / hw + 1; }
-inline uint32_t flat_table_words(uint32_t hw) { return (hw + 1) / 2; }
+inline uint32_t flat_table_words(uint32_t hw) { return (hw + 1) / 2; }            // a 16-bit tile number per position of a plane
+inline uint32_t quad_period(uint32_t hw) { return hw / ((hw & 3u) == 0 ? 4u : (hw & 1u) == 0 ? 2u : 1u); }
+inline uint32_t quad_period_planes(uint32_t hw) { return (hw & 3u) == 0 ? 1u : (hw & 1u) == 0 ? 2u : 4u; }
+inline uint32_t quad_table_words(uint32_t hw) { return 2u * quad_period(hw); }    // 4 16-bit offsets per quad of a period
 inline size_t flat_smem_bytes(uint32_t elems, uint32_t hw, uint32_t tpp) {
-    return 4ull * flat_table_words(hw) + 4ull * flat_planes_per_cta(elems, hw) * tpp;
+    return 4ull * quad_table_words(hw) + 4ull * flat_planes_per_cta(elems, hw) * tpp;
+}
+
+// entry idx of the quad table: for each of the elements 4 idx .. 4 idx + 3 of a run of planes that starts on a
+// plane boundary, (plane inside the run) * TPP + tile inside the plane (fits 16 bits: at most 4 planes of at most
+// FLAT_MAX_HW tiles)
+__device__ __forceinline__ uint2 quad_table_entry(uint32_t idx, uint32_t HW, uint32_t W, uint32_t Wb, uint32_t TPP,
+                                                  const FastDiv& by_hw, const FastDiv& by_w, const FastDiv& by_b) {
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t e = 4u * idx + (uint32_t)i;
+        const uint32_t dp = fdiv(e, by_hw), pos = e - dp * HW;
+        const uint32_t h = fdiv(pos, by_w), w = pos - h * W;
+        o[i] = dp * TPP + fdiv(h, by_b) * Wb + fdiv(w, by_b);
+    }
+    return make_uint2(o[0] | (o[1] << 16), o[2] | (o[3] << 16));
 }
 
 template <typename XT, typename LT, int Q, int QPT>
@@ -251,15 +274,13 @@ __global__ void __launch_bounds__(256)
 decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFlat d) {
     extern __shared__ uint32_t flat_smem[];
-    uint16_t* tile_of = reinterpret_cast<uint16_t*>(flat_smem);      // position inside a plane -> tile inside the plane
+    uint2* quad_of = reinterpret_cast<uint2*>(flat_smem);            // quad inside a period -> where its 4 low-frequency values sit
     float* lfc_s = reinterpret_cast<float*>(flat_smem + d.table_words);   // low-frequency values of this CTA's planes
     __shared__ DeqTable<Q> table;
     const uint32_t n = blockIdx.y;
     table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
-    for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
-        const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
-        tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
-    }
+    for (uint32_t idx = threadIdx.x; idx < d.period; idx += 256u)
+        quad_of[idx] = quad_table_entry(idx, d.HW, d.W, d.Wb, d.TPP, d.by_hw, d.by_w, d.by_b);
     const uint32_t e_first = blockIdx.x * (1024u * QPT);
     const uint32_t plane0 = fdiv(e_first, d.by_hw);
     const uint32_t nplanes = min(d.planes_per_cta, d.C - plane0);
@@ -274,18 +295,15 @@ decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
         if (q < d.qps) {
             const float4 hq = table.quad(quad_bits<Q>(packed, sample_quad0 + q));
             const float hv[4] = {hq.x, hq.y, hq.z, hq.w};
-            const uint32_t plane = fdiv(q * 4u, d.by_hw);
-            uint32_t rem = q * 4u - plane * d.HW;
-            const float* lp = lfc_s + (plane - plane0) * d.TPP;
+            const uint32_t grp = fdiv(q, d.by_period);
+            const uint2 ent = quad_of[q - grp * d.period];
+            // the period may start before the first plane staged here; the elements of this CTA do not
+            const int base = ((int)(grp * d.period_planes) - (int)plane0) * (int)d.TPP;
             float v[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                v[i] = __fadd_rn(lp[tile_of[rem]], hv[i]);
-                if (++rem == d.HW) {
-                    rem = 0;
-                    lp += d.TPP;
-                }
-            }
+            v[0] = __fadd_rn(lfc_s[base + (int)(ent.x & 0xFFFFu)], hv[0]);
+            v[1] = __fadd_rn(lfc_s[base + (int)(ent.x >> 16)], hv[1]);
+            v[2] = __fadd_rn(lfc_s[base + (int)(ent.y & 0xFFFFu)], hv[2]);
+            v[3] = __fadd_rn(lfc_s[base + (int)(ent.y >> 16)], hv[3]);
             Quad<XT>::store(xhat + (sample_quad0 + q) * 4u, v[0], v[1], v[2], v[3]);
         }
     }

@@ -472,7 +472,10 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 d.by_w = make_fastdiv(s.W);
                 d.by_b = make_fastdiv(s.B);
                 const uint32_t per_block = 256u * DEC_QPT;
-                d.table_words = flat_table_words(s.HW);
+                d.table_words = quad_table_words(s.HW);
+                d.period = quad_period(s.HW);
+                d.period_planes = quad_period_planes(s.HW);
+                d.by_period = make_fastdiv(d.period);
                 d.planes_per_cta = flat_planes_per_cta(4u * per_block, s.HW);
                 dim3 grid((d.qps + per_block - 1) / per_block, s.N);
                 decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, flat_smem_bytes(4u * per_block, s.HW, s.TPP), stream>>>(

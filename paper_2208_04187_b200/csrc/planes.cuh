@@ -14,11 +14,11 @@
 // balanced tree, meets the other columns of the tile with xor shuffles (the same tree across columns),
 // and keeps the extremes of its column.
 // plane_quant_kernel: one thread per 4 consecutive elements of the flat sample (they may lie in
-// different tiles, rows or planes): the tile of every position of a plane comes from a table in shared
-// memory, the arithmetic of Eq. 9 runs on packed pairs.
+// different tiles, rows or planes): where their 4 low-frequency values sit comes from the quad table in shared
+// memory (one 8-byte entry per quad of a period of lcm(HW, 4) elements), the arithmetic of Eq. 9 runs on packed pairs.
 #pragma once
 
-#include "decompress.cuh"   // flat_table_words, flat_planes_per_cta, flat_smem_bytes
+#include "decompress.cuh"   // quad table, flat_planes_per_cta, flat_smem_bytes
 #include "fused_v.cuh"
 
 namespace divk {
@@ -29,9 +29,11 @@ struct PlaneGeom {
     uint32_t planes_per_warp;     // 32 / lanes_per_plane
     uint32_t groups;              // ceil(C / planes_per_warp): warp passes per sample
     uint32_t qps;                 // quads per sample = CHW / 4
-    uint32_t table_words;         // 32-bit words the tile table takes in shared memory
+    uint32_t table_words;         // 32-bit words the quad table takes in shared memory
     uint32_t planes_per_cta;      // upper bound of the planes one CTA of the quantise kernel touches
-    FastDiv by_hw, by_w, by_b;
+    uint32_t period;              // quads after which the quad table repeats
+    uint32_t period_planes;       // planes one period covers (1, 2 or 4)
+    FastDiv by_hw, by_w, by_b, by_period;
 };
 
 template <typename XT, typename LT, int P2>
@@ -59,10 +61,8 @@ plane_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
             float sum = tree8<P2>(v);
 #pragma unroll
             for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-            // one lane per tile divides, the others take its result
-            float mean = 0.f;
-            if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
-            mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
+            // after the butterfly every lane of a tile holds the same sum: each divides for itself
+            const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
             const float stored = Elem<LT>::round(mean);
             if (ok) {
                 if (cw == 0) Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
@@ -94,14 +94,12 @@ __global__ void __launch_bounds__(256)
 plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const uint32_t* __restrict__ ws,
                    void* __restrict__ packed_v, float* __restrict__ stats, PlaneGeom g, uint64_t seed) {
     typedef typename PackedUnit<Q>::type OutT;
-    extern __shared__ uint32_t plane_smem[];
-    uint16_t* tile_of = reinterpret_cast<uint16_t*>(plane_smem);          // position inside a plane -> tile inside the plane
+    extern __shared__ __align__(16) uint32_t plane_smem[];
+    uint2* quad_of = reinterpret_cast<uint2*>(plane_smem);                // quad inside a period -> where its 4 low-frequency values sit
     float* lfc_s = reinterpret_cast<float*>(plane_smem + g.table_words);  // stored low-frequency values of this CTA's planes
     const uint32_t n = blockIdx.y;
-    for (uint32_t idx = threadIdx.x; idx < g.HW; idx += 256u) {
-        const uint32_t h = fdiv(idx, g.by_w), w = idx - h * g.W;
-        tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * g.Wb + fdiv(w, g.by_b));
-    }
+    for (uint32_t idx = threadIdx.x; idx < g.period; idx += 256u)
+        quad_of[idx] = quad_table_entry(idx, g.HW, g.W, g.Wb, g.TPP, g.by_hw, g.by_w, g.by_b);
     const uint32_t plane0 = fdiv(blockIdx.x * (1024u * QPT), g.by_hw);
     const uint32_t nplanes = min(g.planes_per_cta, g.C - plane0);
     {
@@ -127,18 +125,12 @@ plane_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const u
         if (q < g.qps) {
             uint64_t xy, zw;
             StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy, zw);
-            const uint32_t plane = fdiv(q * 4u, g.by_hw);
-            uint32_t rem = q * 4u - plane * g.HW;
-            const float* lfc_p = lfc_s + (plane - plane0) * g.TPP;
-            float lf[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                lf[i] = lfc_p[tile_of[rem]];
-                if (++rem == g.HW) {
-                    rem = 0;
-                    lfc_p += g.TPP;
-                }
-            }
+            const uint32_t grp = fdiv(q, g.by_period);
+            const uint2 ent = quad_of[q - grp * g.period];
+            // the period may start before the first plane staged here; the elements of this CTA do not
+            const int lbase = ((int)(grp * g.period_planes) - (int)plane0) * (int)g.TPP;
+            const float lf[4] = {lfc_s[lbase + (int)(ent.x & 0xFFFFu)], lfc_s[lbase + (int)(ent.x >> 16)],
+                                 lfc_s[lbase + (int)(ent.y & 0xFFFFu)], lfc_s[lbase + (int)(ent.y >> 16)]};
             constexpr float qmax = (float)((1 << Q) - 1);
             const uint64_t z = rng_group(base, q);
             uint32_t b0, b1, b2, b3;
@@ -171,18 +163,16 @@ __global__ void __launch_bounds__(256)
 plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, void* __restrict__ packed_v,
                    float* __restrict__ stats, PlaneGeom g, PlaneFused f, uint64_t seed) {
     typedef typename PackedUnit<Q>::type OutT;
-    extern __shared__ uint32_t plane_smem[];
-    uint16_t* tile_of = reinterpret_cast<uint16_t*>(plane_smem);          // position inside a plane -> tile inside the plane
+    extern __shared__ __align__(16) uint32_t plane_smem[];
+    uint2* quad_of = reinterpret_cast<uint2*>(plane_smem);                // quad inside a period -> where its 4 low-frequency values sit
     float* lfc_s = reinterpret_cast<float*>(plane_smem + g.table_words);  // stored low-frequency values of this CTA's planes
     __shared__ uint32_t s_kmin, s_kmax, s_delta, s_scale, s_ok;
     const uint32_t n = blockIdx.y;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t plane0 = blockIdx.x * f.ppc;
     const uint32_t nplanes = plane0 < g.C ? min(f.ppc, g.C - plane0) : 0u;
-    for (uint32_t idx = threadIdx.x; idx < g.HW; idx += 256u) {
-        const uint32_t h = fdiv(idx, g.by_w), w = idx - h * g.W;
-        tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * g.Wb + fdiv(w, g.by_b));
-    }
+    for (uint32_t idx = threadIdx.x; idx < g.period; idx += 256u)
+        quad_of[idx] = quad_table_entry(idx, g.HW, g.W, g.Wb, g.TPP, g.by_hw, g.by_w, g.by_b);
     if (threadIdx.x == 0) {
         s_kmin = 0;
         s_kmax = 0;
@@ -212,9 +202,8 @@ plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
                 float sum = tree8<P2>(v);
 #pragma unroll
                 for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-                float mean = 0.f;
-                if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
-                mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
+                // after the butterfly every lane of a tile holds the same sum: each divides for itself
+                const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
                 const float stored = Elem<LT>::round(mean);
                 if (ok) {
                     if (cw == 0) {
@@ -293,18 +282,12 @@ plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
     for (uint32_t q = qa + threadIdx.x; q < qb; q += 256u) {
         uint64_t xy, zw;
         StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (size_t)q * 4u), xy, zw);
-        const uint32_t plane = fdiv(q * 4u, g.by_hw);
-        uint32_t rem = q * 4u - plane * g.HW;
-        const float* lfc_p = lfc_s + (plane - plane0) * g.TPP;
-        float lf[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            lf[i] = lfc_p[tile_of[rem]];
-            if (++rem == g.HW) {
-                rem = 0;
-                lfc_p += g.TPP;
-            }
-        }
+        const uint32_t grp = fdiv(q, g.by_period);
+        const uint2 ent = quad_of[q - grp * g.period];
+        // the period may start before this CTA's first plane; the elements of this CTA do not
+        const int lbase = ((int)(grp * g.period_planes) - (int)plane0) * (int)g.TPP;
+        const float lf[4] = {lfc_s[lbase + (int)(ent.x & 0xFFFFu)], lfc_s[lbase + (int)(ent.x >> 16)],
+                             lfc_s[lbase + (int)(ent.y & 0xFFFFu)], lfc_s[lbase + (int)(ent.y >> 16)]};
         constexpr float qmax = (float)((1 << Q) - 1);
         const uint64_t z = rng_group(base, q);
         uint32_t b0, b1, b2, b3;
@@ -333,7 +316,10 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
     g.planes_per_warp = 32u / g.lanes_per_plane;
     g.groups = (s.C + g.planes_per_warp - 1) / g.planes_per_warp;
     g.qps = s.CHW / 4;
-    g.table_words = flat_table_words(s.HW);
+    g.table_words = quad_table_words(s.HW);
+    g.period = quad_period(s.HW);
+    g.period_planes = quad_period_planes(s.HW);
+    g.by_period = host_fastdiv(g.period);
     g.planes_per_cta = flat_planes_per_cta(4u * 256u * PLANE_QPT, s.HW);
     if (flat_smem_bytes(4u * 256u * PLANE_QPT, s.HW, s.TPP) > 44000) return false;
     g.by_hw = host_fastdiv(s.HW);
