@@ -25,7 +25,8 @@ namespace divk {
 
 struct PlaneGeom {
     uint32_t C, H, W, B, Hb, Wb, HW, CHW, TPP;
-    uint32_t lanes_per_plane;     // Wb * P2
+    uint32_t cpl;                 // columns a lane of the first half owns: 2 where W and B are even, else 1
+    uint32_t lanes_per_plane;     // Wb * P2 / cpl
     uint32_t planes_per_warp;     // 32 / lanes_per_plane
     uint32_t groups;              // ceil(C / planes_per_warp): warp passes per sample
     uint32_t qps;                 // quads per sample = CHW / 4
@@ -36,42 +37,93 @@ struct PlaneGeom {
     FastDiv by_hw, by_w, by_b, by_period;
 };
 
-template <typename XT, typename LT, int P2>
-__global__ void __launch_bounds__(256)
-plane_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, PlaneGeom g) {
-    const uint32_t n = blockIdx.y;
-    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// One or two adjacent columns of one row, widened to fp32 and packed as a pair (the second half is 0 for one column)
+template <typename XT, int CPL> struct ColLoad;
+template <> struct ColLoad<float, 1> {
+    static __device__ __forceinline__ uint64_t load(const float* p) { return pk2(*p, 0.f); }
+};
+template <> struct ColLoad<float, 2> {
+    static __device__ __forceinline__ uint64_t load(const float* p) { return *reinterpret_cast<const uint64_t*>(p); }
+};
+template <> struct ColLoad<__nv_bfloat16, 1> {
+    static __device__ __forceinline__ uint64_t load(const __nv_bfloat16* p) {
+        return pk2u((uint32_t)*reinterpret_cast<const uint16_t*>(p) << 16, 0u);
+    }
+};
+template <> struct ColLoad<__nv_bfloat16, 2> {
+    static __device__ __forceinline__ uint64_t load(const __nv_bfloat16* p) {
+        const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+        return pk2u(u << 16, u & 0xFFFF0000u);
+    }
+};
+
+// First half for a run of planes: a lane owns CPL adjacent columns of one tile of one plane (P2 / CPL lanes per
+// tile, several planes per warp).  Per band it loads its columns' rows, sums each column with the balanced tree
+// down the rows, meets the tile's other columns (its own second column first, then xor shuffles: the same tree
+// across columns) and keeps the extremes of its columns.  Planes first, first + stride, ... < count of the run at
+// x_run / lfc_run; `keep` (may be null) receives the stored low-frequency values, TPP per plane of the run.
+// Returns the residual extremes of this lane's elements in lo / hi.
+template <typename XT, typename LT, int P2, int CPL>
+__device__ __forceinline__ void plane_half1(const XT* __restrict__ x_run, LT* __restrict__ lfc_run, float* keep, uint32_t first,
+                                            uint32_t stride, uint32_t count, const PlaneGeom& g, uint32_t lane, float& lo,
+                                            float& hi) {
+    constexpr uint32_t LPT = P2 / CPL;                            // lanes per tile
     const uint32_t pl_local = lane / g.lanes_per_plane;
     const uint32_t lw = lane - pl_local * g.lanes_per_plane;
-    const uint32_t bw = lw / P2, cw = lw % P2;
+    const uint32_t bw = lw / LPT, cw = (lw % LPT) * CPL;          // tile column, first own column inside the tile
     const uint32_t cols = (bw < g.Wb) ? min(g.B, g.W - bw * g.B) : 0u;
-    const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
+    const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;     // W and B even where CPL = 2: both columns or none
     const uint32_t col = bw * g.B + cw;
-    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-    for (uint32_t pg = blockIdx.x * 8u + warp; pg < g.groups; pg += gridDim.x * 8u) {
-        const uint32_t plane = pg * g.planes_per_warp + pl_local;
-        const bool ok = lane_ok && plane < g.C;
-        const XT* xp = x + ((size_t)n * g.C + (ok ? plane : 0u)) * g.HW + (ok ? col : 0u);
-        LT* lp = lfc + ((size_t)n * g.C + (ok ? plane : 0u)) * g.TPP + (ok ? bw : 0u);
+    for (uint32_t pp = first; pp < count; pp += stride) {
+        const uint32_t pl = pp + pl_local;
+        const bool ok = lane_ok && pl < count;
+        const XT* xp = x_run + (size_t)(ok ? pl : 0u) * g.HW + (ok ? col : 0u);
+        LT* lp = lfc_run + (size_t)(ok ? pl : 0u) * g.TPP + (ok ? bw : 0u);
         for (uint32_t bh = 0; bh < g.Hb; ++bh) {
-            const uint32_t rows = min(g.B, g.H - bh * g.B);
-            float v[P2];
+            const uint32_t rows = min(g.B, g.H - bh * g.B);       // the same in every lane
+            uint64_t v[P2];
+            if (rows == (uint32_t)P2) {
 #pragma unroll
-            for (int r = 0; r < P2; ++r) v[r] = (ok && (uint32_t)r < rows) ? Elem<XT>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0.f;
-            float sum = tree8<P2>(v);
+                for (int r = 0; r < P2; ++r) v[r] = ok ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0ull;
+            } else {
 #pragma unroll
-            for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+                for (int r = 0; r < P2; ++r)
+                    v[r] = (ok && (uint32_t)r < rows) ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0ull;
+            }
+            uint64_t t[P2];
+#pragma unroll
+            for (int i = 0; i < P2; ++i) t[i] = v[i];
+#pragma unroll
+            for (int w = P2; w > 1; w >>= 1) {
+#pragma unroll
+                for (int i = 0; i < w / 2; ++i) t[i] = add2_rn(t[2 * i], t[2 * i + 1]);
+            }
+            float c0, c1;
+            upk2(t[0], c0, c1);
+            float sum = CPL == 2 ? __fadd_rn(c0, c1) : c0;
+#pragma unroll
+            for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
             // after the butterfly every lane of a tile holds the same sum: each divides for itself
             const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
             const float stored = Elem<LT>::round(mean);
             if (ok) {
-                if (cw == 0) Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
+                if (cw == 0) {
+                    Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
+                    if (keep) keep[pl * g.TPP + bh * g.Wb + bw] = stored;
+                }
                 float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
 #pragma unroll
                 for (int r = 0; r < P2; ++r) {
                     if ((uint32_t)r < rows) {
-                        blo = fminf(blo, v[r]);
-                        bhi = fmaxf(bhi, v[r]);
+                        float a, b;
+                        upk2(v[r], a, b);
+                        if (CPL == 2) {
+                            blo = fmin3(blo, a, b);
+                            bhi = fmax3(bhi, a, b);
+                        } else {
+                            blo = fminf(blo, a);
+                            bhi = fmaxf(bhi, a);
+                        }
                     }
                 }
                 // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
@@ -80,6 +132,17 @@ plane_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
             }
         }
     }
+}
+
+template <typename XT, typename LT, int P2, int CPL>
+__global__ void __launch_bounds__(256)
+plane_stats_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, PlaneGeom g) {
+    const uint32_t n = blockIdx.y;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+    plane_half1<XT, LT, P2, CPL>(x + (size_t)n * g.C * g.HW, lfc + (size_t)n * g.C * g.TPP, nullptr,
+                                 (blockIdx.x * 8u + warp) * g.planes_per_warp, gridDim.x * 8u * g.planes_per_warp, g.C, g, lane,
+                                 lo, hi);
     const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
     const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
     if (lane == 0 && blockIdx.x * 8u + warp < g.groups) {
@@ -158,7 +221,7 @@ struct PlaneFused {
     uint32_t expected;            // arrivals that complete a sample (a test may ask for an unreachable count)
 };
 
-template <typename XT, typename LT, int Q, int P2>
+template <typename XT, typename LT, int Q, int P2, int CPL>
 __global__ void __launch_bounds__(256)
 plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, void* __restrict__ packed_v,
                    float* __restrict__ stats, PlaneGeom g, PlaneFused f, uint64_t seed) {
@@ -180,49 +243,11 @@ plane_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __r
     }
     __syncthreads();
 
-    // ---------------- half 1: a lane owns one tile column of one plane ----------------
+    // ---------------- half 1: a lane owns one or two tile columns of one plane ----------------
     {
-        const uint32_t pl_local = lane / g.lanes_per_plane;
-        const uint32_t lw = lane - pl_local * g.lanes_per_plane;
-        const uint32_t bw = lw / P2, cw = lw % P2;
-        const uint32_t cols = (bw < g.Wb) ? min(g.B, g.W - bw * g.B) : 0u;
-        const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
-        const uint32_t col = bw * g.B + cw;
         float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-        for (uint32_t pp = warp * g.planes_per_warp; pp < nplanes; pp += 8u * g.planes_per_warp) {
-            const uint32_t pl = pp + pl_local;                       // plane inside the CTA's run
-            const bool ok = lane_ok && pl < nplanes;
-            const XT* xp = x + ((size_t)n * g.C + plane0 + (ok ? pl : 0u)) * g.HW + (ok ? col : 0u);
-            LT* lp = lfc + ((size_t)n * g.C + plane0 + (ok ? pl : 0u)) * g.TPP + (ok ? bw : 0u);
-            for (uint32_t bh = 0; bh < g.Hb; ++bh) {
-                const uint32_t rows = min(g.B, g.H - bh * g.B);
-                float v[P2];
-#pragma unroll
-                for (int r = 0; r < P2; ++r) v[r] = (ok && (uint32_t)r < rows) ? Elem<XT>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0.f;
-                float sum = tree8<P2>(v);
-#pragma unroll
-                for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-                // after the butterfly every lane of a tile holds the same sum: each divides for itself
-                const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
-                const float stored = Elem<LT>::round(mean);
-                if (ok) {
-                    if (cw == 0) {
-                        Elem<LT>::store(lp + (size_t)bh * g.Wb, mean);
-                        lfc_s[pl * g.TPP + bh * g.Wb + bw] = stored;
-                    }
-                    float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
-#pragma unroll
-                    for (int r = 0; r < P2; ++r) {
-                        if ((uint32_t)r < rows) {
-                            blo = fminf(blo, v[r]);
-                            bhi = fmaxf(bhi, v[r]);
-                        }
-                    }
-                    lo = fminf(lo, __fsub_rn(blo, stored));
-                    hi = fmaxf(hi, __fsub_rn(bhi, stored));
-                }
-            }
-        }
+        plane_half1<XT, LT, P2, CPL>(x + ((size_t)n * g.C + plane0) * g.HW, lfc + ((size_t)n * g.C + plane0) * g.TPP, lfc_s,
+                                     warp * g.planes_per_warp, 8u * g.planes_per_warp, nplanes, g, lane, lo, hi);
         const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
         const uint32_t kmax = __reduce_max_sync(0xFFFFFFFFu, float_key(hi));
         if (lane == 0) {
@@ -312,7 +337,8 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
     if (s.HW > PLANE_MAX_HW || s.TPP > 65535u || s.N > 65535u) return false;
     PlaneGeom g;
     g.C = s.C; g.H = s.H; g.W = s.W; g.B = s.B; g.Hb = s.Hb; g.Wb = s.Wb; g.HW = s.HW; g.CHW = s.CHW; g.TPP = s.TPP;
-    g.lanes_per_plane = s.Wb * s.P2;
+    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 1u;
+    g.lanes_per_plane = s.Wb * s.P2 / g.cpl;
     g.planes_per_warp = 32u / g.lanes_per_plane;
     g.groups = (s.C + g.planes_per_warp - 1) / g.planes_per_warp;
     g.qps = s.CHW / 4;
@@ -331,17 +357,17 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
 
 // resident CTAs per SM of one instance of the fused kernel with `smem` bytes of dynamic shared memory (asked
 // once per device and size)
-template <typename XT, typename LT, int Q, int P2>
+template <typename XT, typename LT, int Q, int P2, int CPL>
 inline int plane_fused_occupancy(int dev, size_t smem) {
     static SmemSeen cached[DEVICE_CACHE_SLOTS];          // .bytes holds (smem << 8) | count
-    const void* kern = (const void*)plane_fused_kernel<XT, LT, Q, P2>;
+    const void* kern = (const void*)plane_fused_kernel<XT, LT, Q, P2, CPL>;
     const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS && smem < (1u << 22);
     if (slot && cached[dev].fn.load(std::memory_order_acquire) == kern) {
         const int c = cached[dev].bytes.load(std::memory_order_acquire);
         if ((size_t)(c >> 8) == smem && (c & 255) > 0) return c & 255;
     }
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, plane_fused_kernel<XT, LT, Q, P2>, 256, smem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, plane_fused_kernel<XT, LT, Q, P2, CPL>, 256, smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -358,7 +384,7 @@ struct PlaneFusedPlan {
     uint32_t ppc, ctas_per_sample;
     size_t smem;
 };
-template <typename XT, typename LT, int Q, int P2>
+template <typename XT, typename LT, int Q, int P2, int CPL>
 inline bool plan_plane_fused(const Shape& s, const PlaneGeom& g, const DeviceInfo& di, PlaneFusedPlan* out) {
     // planes per CTA: a multiple of 4 (whole quads) and of the planes a warp takes at once; about 8 CTAs per SM in all
     const uint32_t step = 4u / gcd_u32(4u, g.planes_per_warp) * g.planes_per_warp;
@@ -369,7 +395,7 @@ inline bool plan_plane_fused(const Shape& s, const PlaneGeom& g, const DeviceInf
         const uint32_t cps = (s.C + ppc - 1) / ppc;
         const size_t smem = 4ull * g.table_words + 4ull * ppc * s.TPP;
         if (smem > 40000) return false;
-        const int occ = plane_fused_occupancy<XT, LT, Q, P2>(di.dev, smem);
+        const int occ = plane_fused_occupancy<XT, LT, Q, P2, CPL>(di.dev, smem);
         if (occ < 1) return false;
         if ((uint64_t)cps * s.N > (uint64_t)occ * di.sms) {
             if (attempt) return false;
@@ -388,11 +414,11 @@ inline bool plan_plane_fused(const Shape& s, const PlaneGeom& g, const DeviceInf
 }
 
 // launch of the single-launch form; false when it does not apply or the launch was refused
-template <typename XT, typename LT, int Q, int P2>
+template <typename XT, typename LT, int Q, int P2, int CPL>
 inline bool launch_plane_fused(const Shape& s, const div_layout& lo, const PlaneGeom& g, const DeviceInfo& di, const void* x,
                                uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, uint32_t expected, uint64_t timeout_ns) {
     PlaneFusedPlan pf;
-    if (!plan_plane_fused<XT, LT, Q, P2>(s, g, di, &pf)) return false;
+    if (!plan_plane_fused<XT, LT, Q, P2, CPL>(s, g, di, &pf)) return false;
     PlaneFused f;
     f.ppc = pf.ppc;
     f.ctas_per_sample = pf.ctas_per_sample;
@@ -404,7 +430,7 @@ inline bool launch_plane_fused(const Shape& s, const div_layout& lo, const Plane
     float* stats = (float*)(blob + lo.stats_off);
     PlaneGeom gg = g;
     void* args[] = {(void*)&xt, (void*)&lfc, (void*)&ws, (void*)&packed, (void*)&stats, (void*)&gg, (void*)&f, (void*)&seed};
-    if (cudaLaunchCooperativeKernel((const void*)plane_fused_kernel<XT, LT, Q, P2>, dim3(pf.ctas_per_sample, s.N), dim3(256), args,
+    if (cudaLaunchCooperativeKernel((const void*)plane_fused_kernel<XT, LT, Q, P2, CPL>, dim3(pf.ctas_per_sample, s.N), dim3(256), args,
                                     pf.smem, st) != cudaSuccess) {
         cudaGetLastError();
         return false;
@@ -416,7 +442,9 @@ template <typename XT, typename LT>
 inline bool launch_plane_fused_q(int qbits, const Shape& s, const div_layout& lo, const PlaneGeom& g, const DeviceInfo& di,
                                  const void* x, uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st, uint32_t expected,
                                  uint64_t timeout_ns) {
-#define DIVK_PF(QQ, PP) launch_plane_fused<XT, LT, QQ, PP>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns)
+#define DIVK_PF(QQ, PP)                                                                                              \
+    (g.cpl == 2 ? launch_plane_fused<XT, LT, QQ, PP, 2>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns) \
+                : launch_plane_fused<XT, LT, QQ, PP, 1>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns))
     switch (s.P2) {
         case 4: return qbits == 2 ? DIVK_PF(2, 4) : qbits == 4 ? DIVK_PF(4, 4) : DIVK_PF(8, 4);
         case 8: return qbits == 2 ? DIVK_PF(2, 8) : qbits == 4 ? DIVK_PF(4, 8) : DIVK_PF(8, 8);
@@ -431,7 +459,8 @@ inline bool plane_fused_applies(const div_desc* d, const Shape& s, const PlaneGe
     typedef __nv_bfloat16 bf16;
     const DeviceInfo di = device_info();
     if (!di.ok || di.sms < 1) return false;
-#define DIVK_PP(XT, LT, QQ, PP) plan_plane_fused<XT, LT, QQ, PP>(s, g, di, out)
+#define DIVK_PP(XT, LT, QQ, PP) \
+    (g.cpl == 2 ? plan_plane_fused<XT, LT, QQ, PP, 2>(s, g, di, out) : plan_plane_fused<XT, LT, QQ, PP, 1>(s, g, di, out))
 #define DIVK_PQ(XT, LT, PP) (d->qbits == 2 ? DIVK_PP(XT, LT, 2, PP) : d->qbits == 4 ? DIVK_PP(XT, LT, 4, PP) : DIVK_PP(XT, LT, 8, PP))
 #define DIVK_PT(XT, LT) (s.P2 == 4 ? DIVK_PQ(XT, LT, 4) : s.P2 == 8 ? DIVK_PQ(XT, LT, 8) : s.P2 == 16 ? DIVK_PQ(XT, LT, 16) : false)
     if (d->x_dtype == DIV_F32) return d->lfc_dtype == DIV_F32 ? DIVK_PT(float, float) : DIVK_PT(float, bf16);
@@ -458,9 +487,18 @@ inline div_status compress_planes_t(const div_desc* d, const Shape& s, const div
     const XT* xt = (const XT*)x;
     LT* lfc = (LT*)(blob + lo.lfc_off);
     switch (s.P2) {
-        case 4: plane_stats_kernel<XT, LT, 4><<<grid1, 256, 0, st>>>(xt, lfc, ws, g); break;
-        case 8: plane_stats_kernel<XT, LT, 8><<<grid1, 256, 0, st>>>(xt, lfc, ws, g); break;
-        case 16: plane_stats_kernel<XT, LT, 16><<<grid1, 256, 0, st>>>(xt, lfc, ws, g); break;
+        case 4:
+            if (g.cpl == 2) plane_stats_kernel<XT, LT, 4, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 4, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            break;
+        case 8:
+            if (g.cpl == 2) plane_stats_kernel<XT, LT, 8, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 8, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            break;
+        case 16:
+            if (g.cpl == 2) plane_stats_kernel<XT, LT, 16, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 16, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            break;
         default: return DIV_ERR_PARAM;
     }
     if (cudaGetLastError() != cudaSuccess) return DIV_ERR_CUDA;
