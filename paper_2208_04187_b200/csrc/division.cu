@@ -158,6 +158,10 @@ div_status compress_two_pass(const div_desc* d, const Shape& s, const div_layout
 // decompress
 // ------------------------------------------------------------------------------------------
 constexpr int DEC_QPT = 4;
+#ifndef DIVK_FLAT_QPT
+#define DIVK_FLAT_QPT 8
+#endif
+constexpr int FLAT_QPT = DIVK_FLAT_QPT;       // quads per thread of the flat decompress kernel
 
 // Which compress kernels run a descriptor.  Measured on the ResNet / WRN / DenseNet-shaped maps: from about
 // 56 MB up with 8 x 8 blocks the staged kernel is fastest (both reads of x staged through shared memory by bulk
@@ -225,7 +229,7 @@ bool decompress_fast_ok(const Shape& s) {
 }
 bool decompress_flat_ok(const Shape& s) {
     return (s.CHW % 4 == 0) && s.HW <= FLAT_MAX_HW && s.TPP <= 65535 && s.N <= 65535 && s.CHW < (1u << 31) &&
-           flat_smem_bytes(4u * 256u * DEC_QPT, s.HW, s.TPP) <= 40000;
+           flat_smem_bytes(4u * 256u * FLAT_QPT, s.HW, s.TPP) <= 40000;
 }
 
 }  // namespace
@@ -471,14 +475,14 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 d.by_hw = make_fastdiv(s.HW);
                 d.by_w = make_fastdiv(s.W);
                 d.by_b = make_fastdiv(s.B);
-                const uint32_t per_block = 256u * DEC_QPT;
+                const uint32_t per_block = 256u * FLAT_QPT;
                 d.table_words = quad_table_words(s.HW);
                 d.period = quad_period(s.HW);
                 d.period_planes = quad_period_planes(s.HW);
                 d.by_period = make_fastdiv(d.period);
                 d.planes_per_cta = flat_planes_per_cta(4u * per_block, s.HW);
                 dim3 grid((d.qps + per_block - 1) / per_block, s.N);
-                decompress_flat_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, flat_smem_bytes(4u * per_block, s.HW, s.TPP), stream>>>(
+                decompress_flat_kernel<XT, LT, Q, FLAT_QPT><<<grid, 256, flat_smem_bytes(4u * per_block, s.HW, s.TPP), stream>>>(
                     lfc, packed, stats, (XT*)xhat_dev, d);
             } else {
                 const uint64_t g = (nwords + 255) / 256;
