@@ -697,9 +697,9 @@ def run_ours(args):
         pk3, pk3_kind = measured_peak()
         three_d = {"what": "3-D map " + "x".join(map(str, shp)) + f" fp32, B={b3}, Q={q3}, this rank",
                    "compression_ratio": int(lo3.raw_bytes) / int(lo3.closed_form_bytes), "steps": n3,
-                   "compress_kernel": "lfc_stats3d_warp_kernel + quant3d_quad_kernel", "compress_us": round(c_us, 1),
+                   "compress_kernel": "lfc_stats3d_strip_kernel + quant3d_strip_kernel", "compress_us": round(c_us, 1),
                    "compress_GBps": round(b3y / c_us / 1e3, 1), "compress_frac_of_peak": round(b3y / c_us / 1e3 / pk3, 3),
-                   "decompress_kernel": "decompress3d_quad_kernel", "decompress_us": round(d_us, 1),
+                   "decompress_kernel": "decompress3d_strip_kernel", "decompress_us": round(d_us, 1),
                    "decompress_GBps": round(b3y / d_us / 1e3, 1), "decompress_frac_of_peak": round(b3y / d_us / 1e3 / pk3, 3),
                    "peak_kind": f"of {pk3_kind}", "gpu_launches": 3 * (n3 + 3)}
         del pairs3, blob3, ws3

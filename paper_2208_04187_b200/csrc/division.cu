@@ -814,7 +814,15 @@ div_status div_compress_3d(const div_desc3d* desc, const void* x_dev, void* comp
         const uint32_t gpr = bpw ? (s.Wb + bpw - 1u) / bpw : 0u;                       // warp groups per row of blocks
         const uint64_t groups = (uint64_t)s.N * s.C * s.Db * s.Hb * gpr;
         const uint64_t gw = (groups + 7u) / 8u;
-        if (bpw && gw <= 0x7FFFFFFFull) {
+        // W % 4 == 0 and B = 4 or 8: a lane per strip of 4 columns (16-byte loads)
+        const uint64_t strip_slots = (uint64_t)s.N * s.C * s.Db * s.Hb * s.Wb * (s.B / 4u) * 2u;      // two lanes per strip
+        const uint64_t gs = (strip_slots + 127u) / 128u;
+        if (s.W % 4u == 0 && (s.B == 4u || s.B == 8u) && s.P2 == s.B && gs <= 0x7FFFFFFFull) {
+            const XT* xs = (const XT*)x_dev;
+            LT* lf = (LT*)(blob + lo.lfc_off);
+            if (s.B == 8u) lfc_stats3d_strip_kernel<XT, LT, 8><<<(unsigned)gs, 128, 0, stream>>>(xs, lf, ws, s, strip_slots);
+            else lfc_stats3d_strip_kernel<XT, LT, 4><<<(unsigned)gs, 128, 0, stream>>>(xs, lf, ws, s, strip_slots);
+        } else if (bpw && gw <= 0x7FFFFFFFull) {
             const XT* xs = (const XT*)x_dev;
             LT* lf = (LT*)(blob + lo.lfc_off);
             switch (s.P2) {
@@ -829,6 +837,20 @@ div_status div_compress_3d(const div_desc3d* desc, const void* x_dev, void* comp
             lfc_stats3d_kernel<XT, LT><<<(unsigned)g1, 128, 0, stream>>>((const XT*)x_dev, (LT*)(blob + lo.lfc_off), ws, s);
         }
         if (launch_status() != DIV_OK) return DIV_ERR_CUDA;
+        if (s.W % 4u == 0 && (s.B == 4u || s.B == 8u) && s.P2 == s.B && gs <= 0x7FFFFFFFull && desc->qbits != 1) {
+            void* packed = blob + lo.packed_off;
+            float* stats = (float*)(blob + lo.stats_off);
+            const XT* xs = (const XT*)x_dev;
+            const LT* lf = (const LT*)(blob + lo.lfc_off);
+#define DIVK_Q3(QQ, PP) quant3d_strip_kernel<XT, LT, QQ, PP><<<(unsigned)gs, 128, 0, stream>>>(xs, lf, ws, packed, stats, s, seed, strip_slots)
+            if (s.B == 8u) {
+                if (desc->qbits == 2) DIVK_Q3(2, 8); else if (desc->qbits == 4) DIVK_Q3(4, 8); else DIVK_Q3(8, 8);
+            } else {
+                if (desc->qbits == 2) DIVK_Q3(2, 4); else if (desc->qbits == 4) DIVK_Q3(4, 4); else DIVK_Q3(8, 4);
+            }
+#undef DIVK_Q3
+            return launch_status();
+        }
         if (quad3_ok(s) && desc->qbits != 1) {
             const Quad3 g = make_quad3(s);
             const dim3 grid((g.qps + 256u * DEC_QPT - 1) / (256u * DEC_QPT), s.N);
@@ -870,6 +892,22 @@ div_status div_decompress_3d(const div_desc3d* desc, const void* comp_dev, size_
     return dispatch_types(desc->x_dtype, desc->lfc_dtype, [&](auto* xt, auto* lt) -> div_status {
         typedef std::remove_pointer_t<decltype(xt)> XT;
         typedef std::remove_pointer_t<decltype(lt)> LT;
+        // W % 4 == 0, B = 4 or 8, Q in {2,4,8}: a lane per half strip
+        const uint64_t sps = (uint64_t)s.C * s.Db * s.Hb * s.Wb * (s.B / 4u) * 2u;
+        if (s.W % 4u == 0 && (s.B == 4u || s.B == 8u) && s.P2 == s.B && desc->qbits != 1 && sps < (1ull << 31) && s.N <= 65535u) {
+            const dim3 grid((unsigned)((sps + 255u) / 256u), s.N);
+            const LT* lf = (const LT*)(blob + lo.lfc_off);
+            const uint32_t* pk = (const uint32_t*)(blob + lo.packed_off);
+            const float* stt = (const float*)(blob + lo.stats_off);
+#define DIVK_D3(QQ, PP) decompress3d_strip_kernel<XT, LT, QQ, PP><<<grid, 256, 0, stream>>>(lf, pk, stt, (XT*)xhat_dev, s, (uint32_t)sps)
+            if (s.B == 8u) {
+                if (desc->qbits == 2) DIVK_D3(2, 8); else if (desc->qbits == 4) DIVK_D3(4, 8); else DIVK_D3(8, 8);
+            } else {
+                if (desc->qbits == 2) DIVK_D3(2, 4); else if (desc->qbits == 4) DIVK_D3(4, 4); else DIVK_D3(8, 4);
+            }
+#undef DIVK_D3
+            return launch_status();
+        }
         if (quad3_ok(s)) {
             const Quad3 g3 = make_quad3(s);
             const dim3 grid((g3.qps + 256u * DEC_QPT - 1) / (256u * DEC_QPT), s.N);

@@ -119,6 +119,249 @@ lfc_stats3d_warp_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t
     }
 }
 
+// The same for W % 4 == 0 and B = 4 or 8 (the shapes of video and volumetric networks): a lane owns a strip of 4
+// adjacent columns of one block over all its rows and depths (16-byte loads, packed adds), B / 4 lanes per block
+// side by side.  Per row of the block the lane sums its B depth values with the tree, then the B row sums with the
+// same tree, then its 4 columns and, for B = 8, meets the block's other strip by one xor shuffle: the order of
+// lfc_stats3d_kernel.  For more loads in flight the rows of a strip are split between two neighbouring lanes (upper
+// and lower half); their partial sums meet at the top level of the row tree.  Slots are numbered
+// ((vol * Db + bd) * Hb + bh) * (Wb * B / 4 * 2) + 2 * strip in the block row + half; a warp takes 32 consecutive
+// slots (it may straddle block rows, volumes and samples).
+template <typename XT, typename LT, int P2>
+__global__ void __launch_bounds__(128)
+lfc_stats3d_strip_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, Shape3 s, uint64_t slots) {
+    constexpr uint32_t LPB = P2 / 4;                                   // lanes per block
+    const uint32_t lane = threadIdx.x & 31;
+    constexpr uint32_t HR = P2 / 2;                                    // rows per lane
+    const uint64_t slot = (uint64_t)blockIdx.x * 128u + threadIdx.x;          // 4 warps of 32 consecutive slots
+    const uint32_t spr = s.Wb * LPB * 2u;                              // slots per row of blocks
+    const bool live = slot < slots;
+    const uint64_t rowid = (live ? slot : 0ull) / spr;                 // (vol * Db + bd) * Hb + bh
+    const uint32_t sq = (uint32_t)((live ? slot : 0ull) - rowid * spr);
+    const uint32_t half = sq & 1u, strip = sq >> 1;
+    const uint32_t bw = strip / LPB, cw = (strip % LPB) * 4u;
+    const uint64_t vd = rowid / s.Hb;
+    const uint32_t bh = (uint32_t)(rowid - vd * s.Hb);
+    const uint64_t vol = vd / s.Db;
+    const uint32_t bd = (uint32_t)(vd - vol * s.Db);
+    const uint32_t n = (uint32_t)(vol / s.C);
+    const uint32_t d0 = bd * s.B, h0 = bh * s.B, w0 = bw * s.B;
+    const uint32_t nd = min(s.B, s.D - d0), nh = min(s.B, s.H - h0), nw = min(s.B, s.W - w0);
+    const bool ok = live && cw < nw;                                   // W % 4 == 0: a strip is whole or absent
+    const uint32_t r0 = half * HR;                                     // first own row inside the block
+    const XT* base = x + vol * s.DHW + ((size_t)d0 * s.H + h0 + r0) * s.W + (ok ? w0 + cw : 0u);
+    const bool full = __all_sync(0xFFFFFFFFu, !ok || (nd == (uint32_t)P2 && nh == (uint32_t)P2));
+    float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
+    uint64_t txy[4], tzw[4];                                           // partial sums over the rows, one per tree level
+#pragma unroll
+    for (int r = 0; r < (int)HR; ++r) {
+        uint64_t vxy[P2], vzw[P2];
+        // all loads of the row first (they are independent), then the extremes
+        const XT* row = base + (size_t)r * s.W;
+        const size_t plane = (size_t)s.HW;
+        if (full) {
+            if (ok) {
+#pragma unroll
+                for (int k = 0; k < P2; ++k) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(row + k * plane), vxy[k], vzw[k]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < P2; ++k) {
+                    vxy[k] = 0ull;
+                    vzw[k] = 0ull;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < P2; ++k) {
+                vxy[k] = 0ull;
+                vzw[k] = 0ull;
+                if (ok && r0 + (uint32_t)r < nh && (uint32_t)k < nd)
+                    StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(row + k * plane), vxy[k], vzw[k]);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < P2; ++k) {
+            if (ok && (full || (r0 + (uint32_t)r < nh && (uint32_t)k < nd))) {
+                float a, b, c, d;
+                upk2(vxy[k], a, b);
+                upk2(vzw[k], c, d);
+                lo = fmin3(lo, a, b);
+                lo = fmin3(lo, c, d);
+                hi = fmax3(hi, a, b);
+                hi = fmax3(hi, c, d);
+            }
+        }
+#pragma unroll
+        for (int w = P2; w > 1; w >>= 1) {
+#pragma unroll
+            for (int i = 0; i < w / 2; ++i) {
+                vxy[i] = add2_rn(vxy[2 * i], vxy[2 * i + 1]);
+                vzw[i] = add2_rn(vzw[2 * i], vzw[2 * i + 1]);
+            }
+        }
+        // the tree over the rows, neighbours first, kept as one partial sum per level (r is a compile-time
+        // constant here): rows 0+1, 2+3, ... are added as soon as both are there
+        uint64_t cxy = vxy[0], czw = vzw[0];
+        int lv = 0;
+#pragma unroll
+        for (int bit = 1; bit < (int)HR; bit <<= 1) {
+            if (r & bit) {
+                cxy = add2_rn(txy[lv], cxy);
+                czw = add2_rn(tzw[lv], czw);
+                ++lv;
+            } else {
+                break;
+            }
+        }
+        txy[lv] = cxy;
+        tzw[lv] = czw;
+    }
+    constexpr int TOP = P2 == 8 ? 2 : 1;                                // log2(HR): where the sum over the own rows ends up
+    // top level of the row tree: upper half + lower half (the neighbouring lane)
+    const uint64_t sxy = add2_rn(txy[TOP], __shfl_xor_sync(0xFFFFFFFFu, txy[TOP], 1));
+    const uint64_t szw = add2_rn(tzw[TOP], __shfl_xor_sync(0xFFFFFFFFu, tzw[TOP], 1));
+    float c0, c1, c2, c3;
+    upk2(sxy, c0, c1);
+    upk2(szw, c2, c3);
+    float sum = __fadd_rn(__fadd_rn(c0, c1), __fadd_rn(c2, c3));
+    if (LPB == 2u) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, 2));      // an absent strip brings 0
+    uint32_t kmin = 0u, kmax = 0u;                                      // neutral keys
+    if (ok) {
+        const float mean = __fdiv_rn(sum, (float)(nd * nh * nw));
+        const float stored = Elem<LT>::round(mean);
+        if (cw == 0 && half == 0) Elem<LT>::store(lfc + ((vol * s.Db + bd) * s.Hb + bh) * s.Wb + bw, mean);
+        kmin = ~float_key(__fsub_rn(lo, stored));                       // x -> fl(x - stored) is monotone
+        kmax = float_key(__fsub_rn(hi, stored));
+    }
+    // one pair of atomics per warp where the whole warp sits in one sample, else one per lane
+    const uint32_t n0 = __shfl_sync(0xFFFFFFFFu, n, 0);
+    if (__all_sync(0xFFFFFFFFu, !ok || n == n0)) {
+        kmin = __reduce_max_sync(0xFFFFFFFFu, kmin);
+        kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+        if (lane == 0 && (kmin | kmax)) {
+            uint32_t* slot_n = ws + WS_HEADER_WORDS + (size_t)n0 * WS_SLOT_WORDS;
+            atomicMax(slot_n + 0, kmin);
+            atomicMax(slot_n + 1, kmax);
+        }
+    } else if (ok) {
+        uint32_t* slot_n = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+        atomicMax(slot_n + 0, kmin);
+        atomicMax(slot_n + 1, kmax);
+    }
+}
+
+// Quantise half with the same lane-per-strip layout (W % 4 == 0, B = 4 or 8): the lane reads its sample's extremes
+// and its block's stored low-frequency value once, then walks the rows and depths of its strip: per row of 4 elements
+// one 16-byte load, the random word of that group of 4 (the counter advances by a constant per row and per plane),
+// Eq. 9 on packed pairs, one byte / half-word / word of codes.  x is read a second time.
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(128)
+quant3d_strip_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const uint32_t* __restrict__ ws,
+                     void* __restrict__ packed_v, float* __restrict__ stats, Shape3 s, uint64_t seed, uint64_t slots) {
+    typedef typename PackedUnit<Q>::type OutT;
+    constexpr uint32_t LPB = P2 / 4;
+    const uint64_t slot = (uint64_t)blockIdx.x * 128u + threadIdx.x;
+    if (slot >= slots) return;
+    const uint32_t spr = s.Wb * LPB * 2u;                              // two lanes per strip: upper and lower rows
+    const uint64_t rowid = slot / spr;
+    const uint32_t sq = (uint32_t)(slot - rowid * spr);
+    const uint32_t half = sq & 1u, strip = sq >> 1;
+    const uint32_t bw = strip / LPB, cw = (strip % LPB) * 4u;
+    const uint64_t vd = rowid / s.Hb;
+    const uint32_t bh = (uint32_t)(rowid - vd * s.Hb);
+    const uint64_t vol = vd / s.Db;
+    const uint32_t bd = (uint32_t)(vd - vol * s.Db);
+    const uint32_t n = (uint32_t)(vol / s.C);
+    const uint32_t c = (uint32_t)(vol - (uint64_t)n * s.C);
+    const uint32_t d0 = bd * s.B, h0 = bh * s.B, w0 = bw * s.B;
+    const uint32_t nd = min(s.B, s.D - d0), nh = min(s.B, s.H - h0), nw = min(s.B, s.W - w0);
+    const uint32_t* slot_n = ws + WS_HEADER_WORDS + (size_t)n * WS_SLOT_WORDS;
+    const QParams qp = make_qparams(key_float(~__ldg(slot_n + 0)), key_float(__ldg(slot_n + 1)), Q);
+    if (c == 0 && rowid == vol * s.Db * s.Hb && sq == 0) {             // the first slot of the sample
+        stats[2 * (size_t)n + 0] = qp.delta;
+        stats[2 * (size_t)n + 1] = qp.step;
+    }
+    if (cw >= nw) return;                                              // W % 4 == 0: a strip is whole or absent
+    const float stored = Elem<LT>::load(lfc + ((vol * s.Db + bd) * s.Hb + bh) * s.Wb + bw);
+    const uint64_t stored2 = pk2(stored, stored), delta2 = pk2(qp.delta, qp.delta), scale2 = pk2(qp.scale, qp.scale);
+    const uint32_t e0 = c * s.DHW + (d0 * s.H + h0) * s.W + w0 + cw;   // in-sample index of the strip's first element
+    const XT* base = x + (size_t)n * s.CDHW + e0;
+    OutT* out = reinterpret_cast<OutT*>(packed_v) + (((uint64_t)n * s.CDHW + e0) >> 2);
+    const uint32_t W4 = s.W >> 2, HW4 = s.HW >> 2;
+    const uint64_t ctr0 = rng_sample_base(seed, n) + K_GROUP * (uint64_t)((e0 >> 2) + 1u);
+    const uint64_t row_step = K_GROUP * (uint64_t)W4, plane_step = K_GROUP * (uint64_t)HW4;
+    const bool full = nd == (uint32_t)P2;
+    const uint32_t r_end = min(nh, (half + 1u) * (P2 / 2u));
+    for (uint32_t r = half * (P2 / 2u); r < r_end; ++r) {
+        const XT* row = base + (size_t)r * s.W;
+        uint64_t vxy[P2], vzw[P2];
+#pragma unroll
+        for (int k = 0; k < P2; ++k) {
+            vxy[k] = 0ull;
+            vzw[k] = 0ull;
+            if (full || (uint32_t)k < nd) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(row + (size_t)k * s.HW), vxy[k], vzw[k]);
+        }
+        uint64_t ctr = ctr0 + row_step * r;
+        OutT* o = out + (size_t)r * W4;
+#pragma unroll
+        for (int k = 0; k < P2; ++k) {
+            if (full || (uint32_t)k < nd) *o = (OutT)quant_row<Q>(vxy[k], vzw[k], stored2, delta2, scale2, rng_mix(ctr));
+            ctr += plane_step;
+            o += HW4;
+        }
+    }
+}
+
+// Decompress with the lane-per-strip layout (W % 4 == 0, B = 4 or 8, Q in {2,4,8}): the lane reads its block's
+// low-frequency value once, then per row of 4 elements one byte / half-word / word of codes, one look-up in the
+// sample's dequantisation table and one 16-byte (fp32) store.  Two lanes per strip (upper and lower rows).
+// grid = (ceil(slots per sample / 256), N)
+template <typename XT, typename LT, int Q, int P2>
+__global__ void __launch_bounds__(256)
+decompress3d_strip_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed, const float* __restrict__ stats,
+                          XT* __restrict__ xhat, Shape3 s, uint32_t slots_per_sample) {
+    constexpr uint32_t LPB = P2 / 4;
+    __shared__ DeqTable<Q> table;
+    const uint32_t n = blockIdx.y;
+    table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
+    __syncthreads();
+    const uint32_t slot = blockIdx.x * 256u + threadIdx.x;
+    if (slot >= slots_per_sample) return;
+    const uint32_t spr = s.Wb * LPB * 2u;
+    const uint32_t rowid = slot / spr;                                 // (c * Db + bd) * Hb + bh
+    const uint32_t sq = slot - rowid * spr;
+    const uint32_t half = sq & 1u, strip = sq >> 1;
+    const uint32_t bw = strip / LPB, cw = (strip % LPB) * 4u;
+    const uint32_t vd = rowid / s.Hb, bh = rowid - vd * s.Hb;
+    const uint32_t c = vd / s.Db, bd = vd - c * s.Db;
+    const uint32_t d0 = bd * s.B, h0 = bh * s.B, w0 = bw * s.B;
+    const uint32_t nd = min(s.B, s.D - d0), nh = min(s.B, s.H - h0), nw = min(s.B, s.W - w0);
+    if (cw >= nw) return;
+    const float lf = Elem<LT>::load(lfc + (size_t)n * s.C * s.TPV + (size_t)rowid * s.Wb + bw);
+    const uint32_t e0 = c * s.DHW + (d0 * s.H + h0) * s.W + w0 + cw;   // in-sample index of the strip's first element
+    const uint64_t quad0 = ((uint64_t)n * s.CDHW + e0) >> 2;
+    XT* out = xhat + (size_t)n * s.CDHW + e0;
+    const uint32_t W4 = s.W >> 2, HW4 = s.HW >> 2;
+    const bool full = nd == (uint32_t)P2;
+    const uint32_t r_end = min(nh, (half + 1u) * (P2 / 2u));
+    for (uint32_t r = half * (P2 / 2u); r < r_end; ++r) {
+        uint32_t bits[P2];
+#pragma unroll
+        for (int k = 0; k < P2; ++k) {
+            bits[k] = 0u;
+            if (full || (uint32_t)k < nd) bits[k] = quad_bits<Q>(packed, quad0 + (uint64_t)r * W4 + (uint64_t)k * HW4);
+        }
+#pragma unroll
+        for (int k = 0; k < P2; ++k) {
+            if (full || (uint32_t)k < nd) {
+                const float4 hq = table.quad(bits[k]);
+                Quad<XT>::store(out + (size_t)r * s.W + (size_t)k * s.HW, __fadd_rn(lf, hq.x), __fadd_rn(lf, hq.y), __fadd_rn(lf, hq.z),
+                                __fadd_rn(lf, hq.w));
+            }
+        }
+    }
+}
+
 // position of a flat in-sample index
 struct Pos3 {
     uint32_t vol, d, h, w;

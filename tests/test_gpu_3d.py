@@ -48,6 +48,10 @@ CASES = [
     ((2, 8, 16, 28, 28), 8, 2, "f32", "f32"), ((2, 3, 4, 4, 33), 16, 4, "f32", "f32"),
     ((1, 3, 1, 3, 4), 4, 2, "f32", "f32"), ((2, 5, 6, 10, 24), 12, 4, "bf16", "bf16"), ((2, 4, 9, 8, 16), 16, 8, "f32", "f32"),
     ((3, 2, 5, 7, 12), 4, 1, "f32", "f32"), ((1, 2, 40, 12, 8), 8, 2, "f32", "bf16"),
+    # W % 4 == 0 and B in {4, 8}: the strip statistics kernel; ragged depth and height, a last block of 4 columns,
+    # warps that straddle volumes and samples
+    ((3, 5, 6, 10, 12), 4, 2, "f32", "f32"), ((2, 3, 9, 7, 16), 4, 4, "bf16", "bf16"), ((5, 1, 4, 4, 8), 4, 2, "f32", "f32"),
+    ((7, 3, 3, 5, 12), 8, 8, "f32", "bf16"), ((2, 2, 17, 9, 40), 8, 2, "bf16", "f32"),
 ]
 
 
