@@ -191,7 +191,7 @@ void choose_compress(const div_desc* d, const Shape& s, uint32_t flags, Choice* 
     c->code = 0;
     if (two_pass) return;
     if (!(flags & DIV_FLAG_NO_LINE_KERNELS) && plan_lines(d, s, &c->lg)) {
-        c->code = (!(flags & DIV_FLAG_TWO_LAUNCH_PLANES) && line_fused_applies(d, s, &c->lf)) ? 8 : 5;
+        c->code = (!(flags & DIV_FLAG_TWO_LAUNCH_PLANES) && line_fused_applies(d, s, c->lg, &c->lf)) ? 8 : 5;
         return;
     }
     const bool may_staged = !(flags & DIV_FLAG_NO_STAGED_KERNEL);

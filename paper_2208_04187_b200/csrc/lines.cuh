@@ -27,7 +27,12 @@ struct LineGeom {
     float inv_full, inv_tail;   // 1 / count of a full block and of a row's last block when that is a power of two, else 0
     float cnt_full, cnt_tail;
     uint32_t qps;            // quads per sample
-    FastDiv by_cpr, by_qpr;
+    // single-launch kernel: a lane owns a segment of min(B, 16) consecutive elements of one block
+    uint32_t log2B;
+    uint32_t eq;             // quads per segment: 1, 2 or 4
+    uint32_t log2spb;        // log2(segments per block) = log2(B / (4 * eq))
+    uint32_t sps;            // segment slots per row = Wb * segments per block (slots past the row's end are empty)
+    FastDiv by_cpr, by_qpr, by_sps;
 };
 
 constexpr int LINE_U = 4;     // warp chunks a warp works on at a time (their loads are issued together)
@@ -137,7 +142,7 @@ struct LineFused {
     uint64_t timeout_ns;
 };
 
-template <typename XT, typename LT, int Q>
+template <typename XT, typename LT, int Q, int EQ>
 __global__ void __launch_bounds__(256)
 line_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __restrict__ ws, void* __restrict__ packed_v,
                   float* __restrict__ stats, LineGeom g, LineFused f, uint64_t seed) {
@@ -145,7 +150,6 @@ line_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
     __shared__ uint32_t s_kmin, s_kmax, s_delta, s_scale, s_ok;
     const uint32_t n = blockIdx.y;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t lpt = 1u << g.log2lpt;
     const uint32_t row0 = blockIdx.x * f.rpc;
     const uint32_t nrows = row0 < g.C ? min(f.rpc, g.C - row0) : 0u;
     const XT* x_n = x + (size_t)n * g.CHW;
@@ -157,42 +161,61 @@ line_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
     }
     __syncthreads();
 
-    // ---------------- half 1: a lane owns 4 consecutive elements; warp chunks of this CTA's rows ----------------
+    // ---------------- half 1: a lane owns a segment of EQ quads of one block ----------------
+    // Slot j of a row: block j >> log2spb, part j & (spb - 1) of it; the parts of a block sit in neighbouring lanes
+    // (sps is a multiple of spb, which divides 32).  The block sum is the balanced pairwise tree over its positions:
+    // inside the lane over the segment's elements, then by xor shuffles over the parts.
+    const uint32_t spb = 1u << g.log2spb;
+    const uint32_t s0 = row0 * g.sps, s1 = (row0 + nrows) * g.sps;           // this CTA's slots [s0, s1)
     {
-        const uint32_t c0 = row0 * g.cpr, c1 = (row0 + nrows) * g.cpr;       // this CTA's warp chunks [c0, c1)
         float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
-        for (uint32_t wc0 = c0 + warp * LINE_U; wc0 < c1; wc0 += 8u * LINE_U) {
-            uint64_t xy[LINE_U], zw[LINE_U];
-            uint32_t row[LINE_U], q[LINE_U];
-            bool ok[LINE_U];
+        for (uint32_t sb = s0 + warp * 32u; sb < s1; sb += 256u) {
+            const uint32_t sl = sb + lane;
+            const bool live = sl < s1;
+            const uint32_t row = fdiv(live ? sl : s0, g.by_sps);
+            const uint32_t j = (live ? sl : s0) - row * g.sps;
+            const uint32_t t = j >> g.log2spb;                               // block inside the row
+            const uint32_t col = (t << g.log2B) + (j & (spb - 1u)) * (4u * EQ);
+            const uint32_t nq = (live && col < g.W) ? min((uint32_t)EQ, (g.W - col) >> 2) : 0u;
+            const unsigned char* xp = reinterpret_cast<const unsigned char*>(x_n + (row * g.W + (nq ? col : 0u)));
+            uint64_t xy[EQ], zw[EQ];
 #pragma unroll
-            for (int u = 0; u < LINE_U; ++u) {
-                const uint32_t wc = wc0 + u;
-                const bool live = wc < c1;
-                row[u] = fdiv(live ? wc : c0, g.by_cpr);
-                q[u] = ((live ? wc : c0) - row[u] * g.cpr) * 32u + lane;          // quad inside the row
-                ok[u] = live && q[u] < g.qpr;
-                xy[u] = 0ull;
-                zw[u] = 0ull;
-                if (ok[u]) StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + (row[u] * g.W + 4u * q[u])), xy[u], zw[u]);
+            for (int i = 0; i < EQ; ++i) {
+                xy[i] = 0ull;
+                zw[i] = 0ull;
+                if ((uint32_t)i < nq) StripRow2<XT>::load(xp + i * 4 * (int)sizeof(XT), xy[i], zw[i]);
+            }
+            float part[EQ];
+            float blo = 3.402823466e+38f, bhi = -3.402823466e+38f;
+#pragma unroll
+            for (int i = 0; i < EQ; ++i) {
+                float a, b, c, d;
+                upk2(xy[i], a, b);
+                upk2(zw[i], c, d);
+                part[i] = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
+                if ((uint32_t)i < nq) {
+                    blo = fmin3(blo, a, b);
+                    blo = fmin3(blo, c, d);
+                    bhi = fmax3(bhi, a, b);
+                    bhi = fmax3(bhi, c, d);
+                }
             }
 #pragma unroll
-            for (int u = 0; u < LINE_U; ++u) {
-                float a, b, c, d;
-                upk2(xy[u], a, b);
-                upk2(zw[u], c, d);
-                float sum = __fadd_rn(__fadd_rn(a, b), __fadd_rn(c, d));
-                for (uint32_t m = 1; m < lpt; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-                const uint32_t t = q[u] >> g.log2lpt;                         // block inside the row
+            for (int w = EQ; w > 1; w >>= 1) {
+#pragma unroll
+                for (int i = 0; i < w / 2; ++i) part[i] = __fadd_rn(part[2 * i], part[2 * i + 1]);
+            }
+            float sum = part[0];
+            for (uint32_t m = 1; m < spb; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+            if (nq) {
                 const bool tail = t + 1u == g.Wb;
                 const float inv = tail ? g.inv_tail : g.inv_full;
                 const float mean = (inv != 0.f) ? __fmul_rn(sum, inv) : __fdiv_rn(sum, tail ? g.cnt_tail : g.cnt_full);
                 const float stored = Elem<LT>::round(mean);
-                if (ok[u]) {
-                    if ((q[u] & (lpt - 1u)) == 0u) Elem<LT>::store(lfc_n + (row[u] * g.Wb + t), mean);
-                    lo = fminf(lo, __fsub_rn(fminf(fminf(a, b), fminf(c, d)), stored));
-                    hi = fmaxf(hi, __fsub_rn(fmaxf(fmaxf(a, b), fmaxf(c, d)), stored));
-                }
+                if ((j & (spb - 1u)) == 0u) Elem<LT>::store(lfc_n + (row * g.Wb + t), mean);
+                // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
+                lo = fminf(lo, __fsub_rn(blo, stored));
+                hi = fmaxf(hi, __fsub_rn(bhi, stored));
             }
         }
         const uint32_t kmin = __reduce_max_sync(0xFFFFFFFFu, ~float_key(lo));
@@ -244,28 +267,31 @@ line_fused_kernel(const XT* __restrict__ x, LT* __restrict__ lfc, uint32_t* __re
     __syncthreads();
     if (!s_ok || nrows == 0) return;
 
-    // ---------------- half 2: a thread per 4 consecutive elements of the CTA's rows ----------------
+    // ---------------- half 2: the same segments; one low-frequency value and one counter per segment ----------------
     const float delta = __uint_as_float(s_delta), scale = __uint_as_float(s_scale);
     const uint64_t delta2 = pk2(delta, delta), scale2 = pk2(scale, scale);
     const uint64_t base = rng_sample_base(seed, n);
     OutT* packed = reinterpret_cast<OutT*>(packed_v) + (uint64_t)n * g.qps;
-    const uint32_t qa = row0 * g.qpr, qb = (row0 + nrows) * g.qpr;           // this CTA's quads [qa, qb)
-    for (uint32_t q0 = qa + threadIdx.x; q0 < qb; q0 += 256u * 4u) {
-        uint64_t xy[4], zw[4];
-        float lf[4];
+    for (uint32_t sl = s0 + threadIdx.x; sl < s1; sl += 256u) {
+        const uint32_t row = fdiv(sl, g.by_sps);
+        const uint32_t j = sl - row * g.sps;
+        const uint32_t t = j >> g.log2spb;
+        const uint32_t col = (t << g.log2B) + (j & (spb - 1u)) * (4u * EQ);
+        if (col >= g.W) continue;
+        const uint32_t nq = min((uint32_t)EQ, (g.W - col) >> 2);
+        const uint32_t q0 = (row * g.W + col) >> 2;                              // first quad of the segment inside the sample
+        const unsigned char* xp = reinterpret_cast<const unsigned char*>(x_n + (size_t)q0 * 4u);
+        uint64_t xy[EQ], zw[EQ];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t q = q0 + k * 256u;
-            if (q < qb) {
-                StripRow2<XT>::load(reinterpret_cast<const unsigned char*>(x_n + q * 4u), xy[k], zw[k]);
-                const uint32_t row = fdiv(q, g.by_qpr);
-                lf[k] = Elem<LT>::load_cg(lfc_n + (row * g.Wb + ((q - row * g.qpr) >> g.log2lpt)));      // stored by other warps of this CTA
-            }
-        }
+        for (int i = 0; i < EQ; ++i)
+            if ((uint32_t)i < nq) StripRow2<XT>::load(xp + i * 4 * (int)sizeof(XT), xy[i], zw[i]);
+        const float lf = Elem<LT>::load_cg(lfc_n + (row * g.Wb + t));            // stored by this CTA in half 1
+        const uint64_t lf2 = pk2(lf, lf);
+        uint64_t ctr = base + K_GROUP * (uint64_t)(q0 + 1u);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t q = q0 + k * 256u;
-            if (q < qb) packed[q] = (OutT)quant_row<Q>(xy[k], zw[k], pk2(lf[k], lf[k]), delta2, scale2, rng_group(base, q));
+        for (int i = 0; i < EQ; ++i) {
+            if ((uint32_t)i < nq) packed[q0 + i] = (OutT)quant_row<Q>(xy[i], zw[i], lf2, delta2, scale2, rng_mix(ctr));
+            ctr += K_GROUP;
         }
     }
 }
@@ -297,21 +323,28 @@ inline bool plan_lines(const div_desc* d, const Shape& s, LineGeom* out) {
     g.qps = s.CHW / 4;
     g.by_cpr = host_fastdiv(g.cpr);
     g.by_qpr = host_fastdiv(g.qpr);
+    g.log2B = g.log2lpt + 2u;
+    g.eq = s.B >= 16u ? 4u : s.B / 4u;
+    g.log2spb = 0;
+    while (((4u * g.eq) << g.log2spb) < s.B) ++g.log2spb;
+    g.sps = s.Wb << g.log2spb;
+    if ((uint64_t)s.C * g.sps >= (1ull << 31)) return false;
+    g.by_sps = host_fastdiv(g.sps);
     *out = g;
     return true;
 }
 
-template <typename XT, typename LT, int Q>
+template <typename XT, typename LT, int Q, int EQ>
 inline int line_fused_occupancy(int dev) {
     static SmemSeen cached[DEVICE_CACHE_SLOTS];          // .bytes holds the count
-    const void* kern = (const void*)line_fused_kernel<XT, LT, Q>;
+    const void* kern = (const void*)line_fused_kernel<XT, LT, Q, EQ>;
     const bool slot = dev >= 0 && dev < DEVICE_CACHE_SLOTS;
     if (slot && cached[dev].fn.load(std::memory_order_acquire) == kern) {
         const int c = cached[dev].bytes.load(std::memory_order_acquire);
         if (c > 0) return c;
     }
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, line_fused_kernel<XT, LT, Q>, 256, 0) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, line_fused_kernel<XT, LT, Q, EQ>, 256, 0) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -324,9 +357,9 @@ inline int line_fused_occupancy(int dev) {
 }
 
 // rows per CTA and CTAs per sample of the single-launch form; false when its CTAs could not all be resident
-template <typename XT, typename LT, int Q>
+template <typename XT, typename LT, int Q, int EQ>
 inline bool plan_line_fused(const Shape& s, const DeviceInfo& di, LineFused* out) {
-    const int occ = line_fused_occupancy<XT, LT, Q>(di.dev);
+    const int occ = line_fused_occupancy<XT, LT, Q, EQ>(di.dev);
     if (occ < 1) return false;
     const uint64_t capacity = (uint64_t)occ * di.sms;
     if (s.N > capacity) return false;
@@ -341,18 +374,18 @@ inline bool plan_line_fused(const Shape& s, const DeviceInfo& di, LineFused* out
     return true;
 }
 
-template <typename XT, typename LT, int Q>
+template <typename XT, typename LT, int Q, int EQ>
 inline bool launch_line_fused(const Shape& s, const div_layout& lo, const LineGeom& g, const DeviceInfo& di, const void* x,
                               uint8_t* blob, uint32_t* ws, uint64_t seed, cudaStream_t st) {
     LineFused f;
-    if (!plan_line_fused<XT, LT, Q>(s, di, &f)) return false;
+    if (!plan_line_fused<XT, LT, Q, EQ>(s, di, &f)) return false;
     const XT* xt = (const XT*)x;
     LT* lfc = (LT*)(blob + lo.lfc_off);
     void* packed = blob + lo.packed_off;
     float* stats = (float*)(blob + lo.stats_off);
     LineGeom gg = g;
     void* args[] = {(void*)&xt, (void*)&lfc, (void*)&ws, (void*)&packed, (void*)&stats, (void*)&gg, (void*)&f, (void*)&seed};
-    if (cudaLaunchCooperativeKernel((const void*)line_fused_kernel<XT, LT, Q>, dim3(f.ctas_per_sample, s.N), dim3(256), args, 0, st) !=
+    if (cudaLaunchCooperativeKernel((const void*)line_fused_kernel<XT, LT, Q, EQ>, dim3(f.ctas_per_sample, s.N), dim3(256), args, 0, st) !=
         cudaSuccess) {
         cudaGetLastError();
         return false;
@@ -367,12 +400,17 @@ inline div_status compress_lines_t(const div_desc* d, const Shape& s, const div_
     if (!di.ok || di.sms < 1) return DIV_ERR_CUDA;
     if (allow_fused) {
         bool done = false;
+#define DIVK_LF(QQ)                                                                                          \
+    (g.eq == 4 ? launch_line_fused<XT, LT, QQ, 4>(s, lo, g, di, x, blob, ws, seed, st)                        \
+               : g.eq == 2 ? launch_line_fused<XT, LT, QQ, 2>(s, lo, g, di, x, blob, ws, seed, st)            \
+                           : launch_line_fused<XT, LT, QQ, 1>(s, lo, g, di, x, blob, ws, seed, st))
         switch (d->qbits) {
-            case 2: done = launch_line_fused<XT, LT, 2>(s, lo, g, di, x, blob, ws, seed, st); break;
-            case 4: done = launch_line_fused<XT, LT, 4>(s, lo, g, di, x, blob, ws, seed, st); break;
-            case 8: done = launch_line_fused<XT, LT, 8>(s, lo, g, di, x, blob, ws, seed, st); break;
+            case 2: done = DIVK_LF(2); break;
+            case 4: done = DIVK_LF(4); break;
+            case 8: done = DIVK_LF(8); break;
             default: return DIV_ERR_PARAM;
         }
+#undef DIVK_LF
         if (done) return DIV_OK;
     }
     // pass 1: enough CTAs per sample to fill the GPU a few times over, never more than there are warp chunks
@@ -409,14 +447,17 @@ inline div_status compress_lines(const div_desc* d, const Shape& s, const div_la
 }
 
 // would the single-launch form run this descriptor?
-inline bool line_fused_applies(const div_desc* d, const Shape& s, LineFused* out) {
+inline bool line_fused_applies(const div_desc* d, const Shape& s, const LineGeom& g, LineFused* out) {
     typedef __nv_bfloat16 bf16;
     const DeviceInfo di = device_info();
     if (!di.ok || di.sms < 1) return false;
-#define DIVK_LQ(XT, LT) (d->qbits == 2 ? plan_line_fused<XT, LT, 2>(s, di, out) : d->qbits == 4 ? plan_line_fused<XT, LT, 4>(s, di, out) : plan_line_fused<XT, LT, 8>(s, di, out))
+#define DIVK_LE(XT, LT, QQ) \
+    (g.eq == 4 ? plan_line_fused<XT, LT, QQ, 4>(s, di, out) : g.eq == 2 ? plan_line_fused<XT, LT, QQ, 2>(s, di, out) : plan_line_fused<XT, LT, QQ, 1>(s, di, out))
+#define DIVK_LQ(XT, LT) (d->qbits == 2 ? DIVK_LE(XT, LT, 2) : d->qbits == 4 ? DIVK_LE(XT, LT, 4) : DIVK_LE(XT, LT, 8))
     if (d->x_dtype == DIV_F32) return d->lfc_dtype == DIV_F32 ? DIVK_LQ(float, float) : DIVK_LQ(float, bf16);
     return d->lfc_dtype == DIV_F32 ? DIVK_LQ(bf16, float) : DIVK_LQ(bf16, bf16);
 #undef DIVK_LQ
+#undef DIVK_LE
 }
 
 }  // namespace divk
