@@ -18,6 +18,7 @@
 
 #include "decompress.cuh"
 #include "lagged.cuh"
+#include "planes.cuh"     // ColLoad
 
 namespace divk {
 
@@ -239,7 +240,9 @@ struct PgSmall {
     uint64_t seed;
     uint32_t planes;            // N * C
     uint32_t G;                 // planes per CTA; G * HW is a multiple of 4
-    uint32_t lanes_per_plane;   // Wb * P2
+    uint32_t cpl;               // columns a lane of the first half owns: 2 where W and B are even, else 1
+    uint32_t quads_same_plane;  // 1: HW % 4 == 0, the 4 elements of a quad lie in one plane (quad table instead of the tile table)
+    uint32_t lanes_per_plane;   // Wb * P2 / cpl
     uint32_t planes_per_warp;   // 32 / lanes_per_plane
     uint32_t table_words;       // 32-bit words of the tile table
     FastDiv by_hw, by_w, by_b, by_c;
@@ -248,11 +251,11 @@ inline size_t pg_small_smem_bytes(const PgSmall& g) {
     return 4ull * (g.table_words + (size_t)g.G * g.s.TPP + 4ull * g.G);
 }
 
-template <typename XT, typename LT, int Q, int P2>
+template <typename XT, typename LT, int Q, int P2, int CPL>
 __global__ void __launch_bounds__(256)
 pg_small_kernel(const PgSmall g) {
     typedef typename PackedUnit<Q>::type OutT;
-    extern __shared__ uint32_t pg_smem[];
+    extern __shared__ __align__(16) uint32_t pg_smem[];
     const Shape& s = g.s;
     uint16_t* tile_of = reinterpret_cast<uint16_t*>(pg_smem);                 // position in a plane -> tile in the plane
     float* lfc_s = reinterpret_cast<float*>(pg_smem + g.table_words);         // stored low-frequency values, G * TPP
@@ -263,18 +266,25 @@ pg_small_kernel(const PgSmall g) {
     const uint32_t nplanes = min(g.G, g.planes - plane0);
     const XT* x = reinterpret_cast<const XT*>(g.x);
 
-    for (uint32_t idx = tid; idx < s.HW; idx += 256u) {
-        const uint32_t h = fdiv(idx, g.by_w), w = idx - h * s.W;
-        tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * s.Wb + fdiv(w, g.by_b));
+    uint2* quad_of = reinterpret_cast<uint2*>(pg_smem);                       // HW % 4 == 0: quad in a plane -> its 4 tiles
+    if (g.quads_same_plane) {
+        for (uint32_t idx = tid; idx < (s.HW >> 2); idx += 256u)
+            quad_of[idx] = quad_table_entry(idx, s.HW, s.W, s.Wb, s.TPP, g.by_hw, g.by_w, g.by_b);
+    } else {
+        for (uint32_t idx = tid; idx < s.HW; idx += 256u) {
+            const uint32_t h = fdiv(idx, g.by_w), w = idx - h * s.W;
+            tile_of[idx] = (uint16_t)(fdiv(h, g.by_b) * s.Wb + fdiv(w, g.by_b));
+        }
     }
     for (uint32_t i = tid; i < 2u * g.G; i += 256u) s_key[i] = 0u;
     __syncthreads();
 
-    // ---- first half: lane = tile column
+    // ---- first half: lane = CPL adjacent columns of one tile (8-byte loads and packed adds where CPL = 2)
     {
+        constexpr uint32_t LPT = P2 / CPL;                                  // lanes per tile
         const uint32_t pl_local = lane / g.lanes_per_plane;
         const uint32_t lw = lane - pl_local * g.lanes_per_plane;
-        const uint32_t bw = lw / P2, cw = lw % P2;
+        const uint32_t bw = lw / LPT, cw = (lw % LPT) * CPL;
         const uint32_t cols = (bw < s.Wb) ? min(s.B, s.W - bw * s.B) : 0u;
         const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
         const uint32_t col = bw * s.B + cw;
@@ -286,16 +296,25 @@ pg_small_kernel(const PgSmall g) {
             float lo = 3.402823466e+38f, hi = -3.402823466e+38f;
             for (uint32_t bh = 0; bh < s.Hb; ++bh) {
                 const uint32_t rows = min(s.B, s.H - bh * s.B);
-                float v[P2];
+                uint64_t v[P2];
 #pragma unroll
                 for (int r = 0; r < P2; ++r)
-                    v[r] = (ok && (uint32_t)r < rows) ? Elem<XT>::load(xp + (size_t)(bh * s.B + r) * s.W) : 0.f;
-                float sum = tree8<P2>(v);
+                    v[r] = (ok && (uint32_t)r < rows) ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * s.B + r) * s.W) : 0ull;
+                uint64_t t[P2];
 #pragma unroll
-                for (int m = 1; m < P2; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
-                float mean = 0.f;
-                if (cw == 0) mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));      // one lane per tile divides
-                mean = __shfl_sync(0xFFFFFFFFu, mean, (int)(lane - cw));
+                for (int i = 0; i < P2; ++i) t[i] = v[i];
+#pragma unroll
+                for (int w = P2; w > 1; w >>= 1) {
+#pragma unroll
+                    for (int i = 0; i < w / 2; ++i) t[i] = add2_rn(t[2 * i], t[2 * i + 1]);
+                }
+                float c0, c1;
+                upk2(t[0], c0, c1);
+                float sum = CPL == 2 ? __fadd_rn(c0, c1) : c0;
+#pragma unroll
+                for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
+                // after the butterfly every lane of a tile holds the same sum: each divides for itself
+                const float mean = __fdiv_rn(sum, (float)(rows * max(cols, 1u)));
                 const float stored = Elem<LT>::round(mean);
                 if (ok) {
                     if (cw == 0) {
@@ -306,8 +325,15 @@ pg_small_kernel(const PgSmall g) {
 #pragma unroll
                     for (int r = 0; r < P2; ++r) {
                         if ((uint32_t)r < rows) {
-                            blo = fminf(blo, v[r]);
-                            bhi = fmaxf(bhi, v[r]);
+                            float a, b;
+                            upk2(v[r], a, b);
+                            if (CPL == 2) {
+                                blo = fmin3(blo, a, b);
+                                bhi = fmax3(bhi, a, b);
+                            } else {
+                                blo = fminf(blo, a);
+                                bhi = fmaxf(bhi, a);
+                            }
                         }
                     }
                     // x -> fl(x - stored) is monotone: the residual extremes are those of the extreme x
@@ -318,7 +344,7 @@ pg_small_kernel(const PgSmall g) {
             // the columns of one tile meet through shuffles, the tiles of one plane in shared memory
             uint32_t kmin = ~float_key(lo), kmax = float_key(hi);
 #pragma unroll
-            for (int m = 1; m < P2; m <<= 1) {
+            for (int m = 1; m < (int)LPT; m <<= 1) {
                 kmin = max(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, m));
                 kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, m));
             }
@@ -354,14 +380,30 @@ pg_small_kernel(const PgSmall g) {
             const uint32_t n = fdiv(plane, g.by_c);
             const uint32_t e = (plane - n * s.C) * s.HW + rem;             // in-sample index of the first element
             float lf[4], dl[4], sc[4];
+            if (g.quads_same_plane) {
+                // one 8-byte entry holds the 4 tiles; one pair of parameters for the quad
+                const uint2 ent = quad_of[rem >> 2];
+                const float* lp = lfc_s + pc * s.TPP;
+                lf[0] = lp[ent.x & 0xFFFFu];
+                lf[1] = lp[ent.x >> 16];
+                lf[2] = lp[ent.y & 0xFFFFu];
+                lf[3] = lp[ent.y >> 16];
+                const float d0 = s_par[2u * pc], s0 = s_par[2u * pc + 1u];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                lf[i] = lfc_s[pc * s.TPP + tile_of[rem]];
-                dl[i] = s_par[2u * pc];
-                sc[i] = s_par[2u * pc + 1u];
-                if (++rem == s.HW) {
-                    rem = 0;
-                    ++pc;
+                for (int i = 0; i < 4; ++i) {
+                    dl[i] = d0;
+                    sc[i] = s0;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    lf[i] = lfc_s[pc * s.TPP + tile_of[rem]];
+                    dl[i] = s_par[2u * pc];
+                    sc[i] = s_par[2u * pc + 1u];
+                    if (++rem == s.HW) {
+                        rem = 0;
+                        ++pc;
+                    }
                 }
             }
             const uint64_t z = rng_group(rng_sample_base(g.seed, n), e >> 2);
@@ -540,7 +582,7 @@ __global__ void __launch_bounds__(256)
 pg_decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                           const uint32_t* __restrict__ stats, XT* __restrict__ xhat, PgDecFlat d) {
     constexpr uint32_t MASK = (1u << Q) - 1u;
-    extern __shared__ uint32_t pg_smem[];
+    extern __shared__ __align__(16) uint32_t pg_smem[];
     uint16_t* tile_of = reinterpret_cast<uint16_t*>(pg_smem);
     for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
         const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
@@ -675,7 +717,9 @@ inline bool plan_pg_small(const div_desc* d, const Shape& s, PgSmall* out) {
     PgSmall g;
     g.s = s;
     g.planes = (uint32_t)planes;
-    g.lanes_per_plane = s.Wb * s.P2;
+    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 1u;
+    g.quads_same_plane = (s.HW % 4 == 0) ? 1u : 0u;
+    g.lanes_per_plane = s.Wb * s.P2 / g.cpl;
     g.planes_per_warp = 32u / g.lanes_per_plane;
     // planes per CTA: whole passes of the 8 warps (a multiple of 8, so G * HW is a multiple of 4), about 8192
     // elements, bounded so that the per-plane arrays stay small
@@ -700,7 +744,11 @@ inline div_status launch_pg_small(int qbits, uint32_t p2, const PgSmall& g, cuda
     const uint32_t grid = (g.planes + g.G - 1) / g.G;
     const size_t smem = pg_small_smem_bytes(g);
 #define DIVK_PGS_CASE(QQ, PP) \
-    if (qbits == QQ && p2 == PP) { pg_small_kernel<XT, LT, QQ, PP><<<grid, 256, smem, st>>>(g); return DIV_OK; }
+    if (qbits == QQ && p2 == PP) {                                                      \
+        if (g.cpl == 2) pg_small_kernel<XT, LT, QQ, PP, 2><<<grid, 256, smem, st>>>(g); \
+        else pg_small_kernel<XT, LT, QQ, PP, 1><<<grid, 256, smem, st>>>(g);            \
+        return DIV_OK;                                                                  \
+    }
     DIVK_PGS_CASE(2, 4)
     DIVK_PGS_CASE(4, 4)
     DIVK_PGS_CASE(8, 4)
