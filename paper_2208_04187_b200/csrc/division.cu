@@ -679,6 +679,7 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
                 d.Wb = s.Wb;
                 d.TPP = s.TPP;
                 d.table_words = flat_table_words(s.HW);
+                d.quads_same_plane = (s.HW % 4u == 0) ? 1u : 0u;
                 d.by_hw = make_fastdiv(s.HW);
                 d.by_w = make_fastdiv(s.W);
                 d.by_b = make_fastdiv(s.B);

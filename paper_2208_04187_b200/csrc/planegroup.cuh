@@ -575,6 +575,7 @@ struct PgDecFlat {
     uint64_t quads;          // N*C*H*W / 4
     uint32_t HW, W, Wb, TPP;
     uint32_t table_words;
+    uint32_t quads_same_plane;   // 1: HW % 4 == 0, a quad lies in one plane (quad table, one pair of parameters per quad)
     FastDiv by_hw, by_w, by_b;
 };
 template <typename XT, typename LT, int Q, int QPT>
@@ -584,9 +585,15 @@ pg_decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict
     constexpr uint32_t MASK = (1u << Q) - 1u;
     extern __shared__ __align__(16) uint32_t pg_smem[];
     uint16_t* tile_of = reinterpret_cast<uint16_t*>(pg_smem);
-    for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
-        const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
-        tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
+    uint2* quad_of = reinterpret_cast<uint2*>(pg_smem);
+    if (d.quads_same_plane) {
+        for (uint32_t idx = threadIdx.x; idx < (d.HW >> 2); idx += 256u)
+            quad_of[idx] = quad_table_entry(idx, d.HW, d.W, d.Wb, d.TPP, d.by_hw, d.by_w, d.by_b);
+    } else {
+        for (uint32_t idx = threadIdx.x; idx < d.HW; idx += 256u) {
+            const uint32_t h = fdiv(idx, d.by_w), w = idx - h * d.W;
+            tile_of[idx] = (uint16_t)(fdiv(h, d.by_b) * d.Wb + fdiv(w, d.by_b));
+        }
     }
     __syncthreads();
     const uint64_t cta_e0 = (uint64_t)blockIdx.x * (1024u * QPT);           // first element of this CTA
@@ -603,15 +610,26 @@ pg_decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict
             uint32_t rem = loc - dp * d.HW;
             uint64_t plane = cta_plane0 + dp;
             float v[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            if (d.quads_same_plane) {
                 float delta, step;
                 pg_unpack_stats(__ldg(stats + plane), delta, step);
-                const float l = Elem<LT>::load(lfc + plane * d.TPP + tile_of[rem]);
-                v[i] = reconstruct((bits >> (i * Q)) & MASK, step, delta, l);
-                if (++rem == d.HW) {
-                    rem = 0;
-                    ++plane;
+                const uint2 ent = quad_of[rem >> 2];
+                const LT* lp = lfc + plane * d.TPP;
+                v[0] = reconstruct(bits & MASK, step, delta, Elem<LT>::load(lp + (ent.x & 0xFFFFu)));
+                v[1] = reconstruct((bits >> Q) & MASK, step, delta, Elem<LT>::load(lp + (ent.x >> 16)));
+                v[2] = reconstruct((bits >> (2 * Q)) & MASK, step, delta, Elem<LT>::load(lp + (ent.y & 0xFFFFu)));
+                v[3] = reconstruct((bits >> (3 * Q)) & MASK, step, delta, Elem<LT>::load(lp + (ent.y >> 16)));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float delta, step;
+                    pg_unpack_stats(__ldg(stats + plane), delta, step);
+                    const float l = Elem<LT>::load(lfc + plane * d.TPP + tile_of[rem]);
+                    v[i] = reconstruct((bits >> (i * Q)) & MASK, step, delta, l);
+                    if (++rem == d.HW) {
+                        rem = 0;
+                        ++plane;
+                    }
                 }
             }
             Quad<XT>::store(xhat + gq * 4u, v[0], v[1], v[2], v[3]);
