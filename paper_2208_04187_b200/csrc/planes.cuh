@@ -25,8 +25,8 @@ namespace divk {
 
 struct PlaneGeom {
     uint32_t C, H, W, B, Hb, Wb, HW, CHW, TPP;
-    uint32_t cpl;                 // columns a lane of the first half owns: 2 where W and B are even, else 1
-    uint32_t lanes_per_plane;     // Wb * P2 / cpl
+    uint32_t cpl;                 // first half, how a lane reads its 2 adjacent columns: 2 = one 8-byte load (W and B even), 3 = two loads
+    uint32_t lanes_per_plane;     // Wb * P2 / 2
     uint32_t planes_per_warp;     // 32 / lanes_per_plane
     uint32_t groups;              // ceil(C / planes_per_warp): warp passes per sample
     uint32_t qps;                 // quads per sample = CHW / 4
@@ -57,8 +57,22 @@ template <> struct ColLoad<__nv_bfloat16, 2> {
     }
 };
 
-// First half for a run of planes: a lane owns CPL adjacent columns of one tile of one plane (P2 / CPL lanes per
-// tile, several planes per warp).  Per band it loads its columns' rows, sums each column with the balanced tree
+// the lane's columns of one row: CPL 1 one column, 2 two columns by one aligned load, 3 two columns by two loads
+// (the second only where it exists)
+template <typename XT, int CPL>
+__device__ __forceinline__ uint64_t load_cols(const XT* p, bool second) {
+    if (CPL == 3) {
+        float a, b, z;
+        upk2(ColLoad<XT, 1>::load(p), a, z);
+        b = 0.f;
+        if (second) upk2(ColLoad<XT, 1>::load(p + 1), b, z);
+        return pk2(a, b);
+    }
+    return ColLoad<XT, CPL == 3 ? 1 : CPL>::load(p);
+}
+
+// First half for a run of planes: a lane owns two adjacent columns of one tile of one plane (P2 / 2 lanes per
+// tile, several planes per warp; CPL says how they are loaded, see load_cols).  Per band it loads its columns' rows, sums each column with the balanced tree
 // down the rows, meets the tile's other columns (its own second column first, then xor shuffles: the same tree
 // across columns) and keeps the extremes of its columns.  Planes first, first + stride, ... < count of the run at
 // x_run / lfc_run; `keep` (may be null) receives the stored low-frequency values, TPP per plane of the run.
@@ -67,12 +81,14 @@ template <typename XT, typename LT, int P2, int CPL>
 __device__ __forceinline__ void plane_half1(const XT* __restrict__ x_run, LT* __restrict__ lfc_run, float* keep, uint32_t first,
                                             uint32_t stride, uint32_t count, const PlaneGeom& g, uint32_t lane, float& lo,
                                             float& hi) {
-    constexpr uint32_t LPT = P2 / CPL;                            // lanes per tile
+    constexpr uint32_t NC = CPL == 1 ? 1u : 2u;                   // columns per lane (CPL 2: one 8-byte load, 3: two loads)
+    constexpr uint32_t LPT = P2 / NC;                             // lanes per tile
     const uint32_t pl_local = lane / g.lanes_per_plane;
     const uint32_t lw = lane - pl_local * g.lanes_per_plane;
-    const uint32_t bw = lw / LPT, cw = (lw % LPT) * CPL;          // tile column, first own column inside the tile
+    const uint32_t bw = lw / LPT, cw = (lw % LPT) * NC;           // tile column, first own column inside the tile
     const uint32_t cols = (bw < g.Wb) ? min(g.B, g.W - bw * g.B) : 0u;
     const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;     // W and B even where CPL = 2: both columns or none
+    const bool second = cw + 1u < cols;                                  // CPL = 3: the second column may lie past the tile's edge
     const uint32_t col = bw * g.B + cw;
     for (uint32_t pp = first; pp < count; pp += stride) {
         const uint32_t pl = pp + pl_local;
@@ -84,11 +100,11 @@ __device__ __forceinline__ void plane_half1(const XT* __restrict__ x_run, LT* __
             uint64_t v[P2];
             if (rows == (uint32_t)P2) {
 #pragma unroll
-                for (int r = 0; r < P2; ++r) v[r] = ok ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0ull;
+                for (int r = 0; r < P2; ++r) v[r] = ok ? load_cols<XT, CPL>(xp + (size_t)(bh * g.B + r) * g.W, second) : 0ull;
             } else {
 #pragma unroll
                 for (int r = 0; r < P2; ++r)
-                    v[r] = (ok && (uint32_t)r < rows) ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * g.B + r) * g.W) : 0ull;
+                    v[r] = (ok && (uint32_t)r < rows) ? load_cols<XT, CPL>(xp + (size_t)(bh * g.B + r) * g.W, second) : 0ull;
             }
             uint64_t t[P2];
 #pragma unroll
@@ -100,7 +116,7 @@ __device__ __forceinline__ void plane_half1(const XT* __restrict__ x_run, LT* __
             }
             float c0, c1;
             upk2(t[0], c0, c1);
-            float sum = CPL == 2 ? __fadd_rn(c0, c1) : c0;
+            float sum = NC == 2 ? __fadd_rn(c0, c1) : c0;              // an absent second column brings the zero it stands for
 #pragma unroll
             for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
             // after the butterfly every lane of a tile holds the same sum: each divides for itself
@@ -117,7 +133,7 @@ __device__ __forceinline__ void plane_half1(const XT* __restrict__ x_run, LT* __
                     if ((uint32_t)r < rows) {
                         float a, b;
                         upk2(v[r], a, b);
-                        if (CPL == 2) {
+                        if (CPL == 2 || (CPL == 3 && second)) {
                             blo = fmin3(blo, a, b);
                             bhi = fmax3(bhi, a, b);
                         } else {
@@ -337,8 +353,8 @@ inline bool plan_planes(const div_desc* d, const Shape& s, PlaneGeom* out) {
     if (s.HW > PLANE_MAX_HW || s.TPP > 65535u || s.N > 65535u) return false;
     PlaneGeom g;
     g.C = s.C; g.H = s.H; g.W = s.W; g.B = s.B; g.Hb = s.Hb; g.Wb = s.Wb; g.HW = s.HW; g.CHW = s.CHW; g.TPP = s.TPP;
-    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 1u;
-    g.lanes_per_plane = s.Wb * s.P2 / g.cpl;
+    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 3u;
+    g.lanes_per_plane = s.Wb * s.P2 / 2u;
     g.planes_per_warp = 32u / g.lanes_per_plane;
     g.groups = (s.C + g.planes_per_warp - 1) / g.planes_per_warp;
     g.qps = s.CHW / 4;
@@ -444,7 +460,7 @@ inline bool launch_plane_fused_q(int qbits, const Shape& s, const div_layout& lo
                                  uint64_t timeout_ns) {
 #define DIVK_PF(QQ, PP)                                                                                              \
     (g.cpl == 2 ? launch_plane_fused<XT, LT, QQ, PP, 2>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns) \
-                : launch_plane_fused<XT, LT, QQ, PP, 1>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns))
+                : launch_plane_fused<XT, LT, QQ, PP, 3>(s, lo, g, di, x, blob, ws, seed, st, expected, timeout_ns))
     switch (s.P2) {
         case 4: return qbits == 2 ? DIVK_PF(2, 4) : qbits == 4 ? DIVK_PF(4, 4) : DIVK_PF(8, 4);
         case 8: return qbits == 2 ? DIVK_PF(2, 8) : qbits == 4 ? DIVK_PF(4, 8) : DIVK_PF(8, 8);
@@ -460,7 +476,7 @@ inline bool plane_fused_applies(const div_desc* d, const Shape& s, const PlaneGe
     const DeviceInfo di = device_info();
     if (!di.ok || di.sms < 1) return false;
 #define DIVK_PP(XT, LT, QQ, PP) \
-    (g.cpl == 2 ? plan_plane_fused<XT, LT, QQ, PP, 2>(s, g, di, out) : plan_plane_fused<XT, LT, QQ, PP, 1>(s, g, di, out))
+    (g.cpl == 2 ? plan_plane_fused<XT, LT, QQ, PP, 2>(s, g, di, out) : plan_plane_fused<XT, LT, QQ, PP, 3>(s, g, di, out))
 #define DIVK_PQ(XT, LT, PP) (d->qbits == 2 ? DIVK_PP(XT, LT, 2, PP) : d->qbits == 4 ? DIVK_PP(XT, LT, 4, PP) : DIVK_PP(XT, LT, 8, PP))
 #define DIVK_PT(XT, LT) (s.P2 == 4 ? DIVK_PQ(XT, LT, 4) : s.P2 == 8 ? DIVK_PQ(XT, LT, 8) : s.P2 == 16 ? DIVK_PQ(XT, LT, 16) : false)
     if (d->x_dtype == DIV_F32) return d->lfc_dtype == DIV_F32 ? DIVK_PT(float, float) : DIVK_PT(float, bf16);
@@ -489,15 +505,15 @@ inline div_status compress_planes_t(const div_desc* d, const Shape& s, const div
     switch (s.P2) {
         case 4:
             if (g.cpl == 2) plane_stats_kernel<XT, LT, 4, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
-            else plane_stats_kernel<XT, LT, 4, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 4, 3><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
             break;
         case 8:
             if (g.cpl == 2) plane_stats_kernel<XT, LT, 8, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
-            else plane_stats_kernel<XT, LT, 8, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 8, 3><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
             break;
         case 16:
             if (g.cpl == 2) plane_stats_kernel<XT, LT, 16, 2><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
-            else plane_stats_kernel<XT, LT, 16, 1><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
+            else plane_stats_kernel<XT, LT, 16, 3><<<grid1, 256, 0, st>>>(xt, lfc, ws, g);
             break;
         default: return DIV_ERR_PARAM;
     }
