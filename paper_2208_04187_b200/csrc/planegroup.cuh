@@ -240,9 +240,9 @@ struct PgSmall {
     uint64_t seed;
     uint32_t planes;            // N * C
     uint32_t G;                 // planes per CTA; G * HW is a multiple of 4
-    uint32_t cpl;               // columns a lane of the first half owns: 2 where W and B are even, else 1
+    uint32_t cpl;               // first half, how a lane reads its 2 adjacent columns: 2 = one 8-byte load (W and B even), 3 = two loads
     uint32_t quads_same_plane;  // 1: HW % 4 == 0, the 4 elements of a quad lie in one plane (quad table instead of the tile table)
-    uint32_t lanes_per_plane;   // Wb * P2 / cpl
+    uint32_t lanes_per_plane;   // Wb * P2 / 2
     uint32_t planes_per_warp;   // 32 / lanes_per_plane
     uint32_t table_words;       // 32-bit words of the tile table
     FastDiv by_hw, by_w, by_b, by_c;
@@ -279,14 +279,16 @@ pg_small_kernel(const PgSmall g) {
     for (uint32_t i = tid; i < 2u * g.G; i += 256u) s_key[i] = 0u;
     __syncthreads();
 
-    // ---- first half: lane = CPL adjacent columns of one tile (8-byte loads and packed adds where CPL = 2)
+    // ---- first half: lane = two adjacent columns of one tile (packed adds; CPL says how they are loaded, see load_cols)
     {
-        constexpr uint32_t LPT = P2 / CPL;                                  // lanes per tile
+        constexpr uint32_t NC = CPL == 1 ? 1u : 2u;
+        constexpr uint32_t LPT = P2 / NC;                                   // lanes per tile
         const uint32_t pl_local = lane / g.lanes_per_plane;
         const uint32_t lw = lane - pl_local * g.lanes_per_plane;
-        const uint32_t bw = lw / LPT, cw = (lw % LPT) * CPL;
+        const uint32_t bw = lw / LPT, cw = (lw % LPT) * NC;
         const uint32_t cols = (bw < s.Wb) ? min(s.B, s.W - bw * s.B) : 0u;
         const bool lane_ok = pl_local < g.planes_per_warp && cw < cols;
+        const bool second = cw + 1u < cols;
         const uint32_t col = bw * s.B + cw;
         for (uint32_t pp = warp; pp * g.planes_per_warp < nplanes; pp += 8u) {
             const uint32_t pc = pp * g.planes_per_warp + pl_local;          // plane inside the CTA
@@ -299,7 +301,7 @@ pg_small_kernel(const PgSmall g) {
                 uint64_t v[P2];
 #pragma unroll
                 for (int r = 0; r < P2; ++r)
-                    v[r] = (ok && (uint32_t)r < rows) ? ColLoad<XT, CPL>::load(xp + (size_t)(bh * s.B + r) * s.W) : 0ull;
+                    v[r] = (ok && (uint32_t)r < rows) ? load_cols<XT, CPL>(xp + (size_t)(bh * s.B + r) * s.W, second) : 0ull;
                 uint64_t t[P2];
 #pragma unroll
                 for (int i = 0; i < P2; ++i) t[i] = v[i];
@@ -310,7 +312,7 @@ pg_small_kernel(const PgSmall g) {
                 }
                 float c0, c1;
                 upk2(t[0], c0, c1);
-                float sum = CPL == 2 ? __fadd_rn(c0, c1) : c0;
+                float sum = NC == 2 ? __fadd_rn(c0, c1) : c0;
 #pragma unroll
                 for (int m = 1; m < (int)LPT; m <<= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xFFFFFFFFu, sum, m));
                 // after the butterfly every lane of a tile holds the same sum: each divides for itself
@@ -327,7 +329,7 @@ pg_small_kernel(const PgSmall g) {
                         if ((uint32_t)r < rows) {
                             float a, b;
                             upk2(v[r], a, b);
-                            if (CPL == 2) {
+                            if (CPL == 2 || (CPL == 3 && second)) {
                                 blo = fmin3(blo, a, b);
                                 bhi = fmax3(bhi, a, b);
                             } else {
@@ -735,9 +737,9 @@ inline bool plan_pg_small(const div_desc* d, const Shape& s, PgSmall* out) {
     PgSmall g;
     g.s = s;
     g.planes = (uint32_t)planes;
-    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 1u;
+    g.cpl = (s.W % 2 == 0 && s.B % 2 == 0) ? 2u : 3u;
     g.quads_same_plane = (s.HW % 4 == 0) ? 1u : 0u;
-    g.lanes_per_plane = s.Wb * s.P2 / g.cpl;
+    g.lanes_per_plane = s.Wb * s.P2 / 2u;
     g.planes_per_warp = 32u / g.lanes_per_plane;
     // planes per CTA: whole passes of the 8 warps (a multiple of 8, so G * HW is a multiple of 4), about 8192
     // elements, bounded so that the per-plane arrays stay small
@@ -764,7 +766,7 @@ inline div_status launch_pg_small(int qbits, uint32_t p2, const PgSmall& g, cuda
 #define DIVK_PGS_CASE(QQ, PP) \
     if (qbits == QQ && p2 == PP) {                                                      \
         if (g.cpl == 2) pg_small_kernel<XT, LT, QQ, PP, 2><<<grid, 256, smem, st>>>(g); \
-        else pg_small_kernel<XT, LT, QQ, PP, 1><<<grid, 256, smem, st>>>(g);            \
+        else pg_small_kernel<XT, LT, QQ, PP, 3><<<grid, 256, smem, st>>>(g);            \
         return DIV_OK;                                                                  \
     }
     DIVK_PGS_CASE(2, 4)
