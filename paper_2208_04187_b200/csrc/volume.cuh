@@ -260,8 +260,10 @@ quant3d_strip_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const
                      void* __restrict__ packed_v, float* __restrict__ stats, Shape3 s, uint64_t seed, uint64_t slots) {
     typedef typename PackedUnit<Q>::type OutT;
     constexpr uint32_t LPB = P2 / 4;
-    const uint64_t slot = (uint64_t)blockIdx.x * 128u + threadIdx.x;
-    if (slot >= slots) return;
+    // slots are taken from the end of the tensor backwards: what the statistics kernel read last is still in the L2
+    const uint64_t back = (uint64_t)blockIdx.x * 128u + threadIdx.x;
+    if (back >= slots) return;
+    const uint64_t slot = slots - 1u - back;
     const uint32_t spr = s.Wb * LPB * 2u;                              // two lanes per strip: upper and lower rows
     const uint64_t rowid = slot / spr;
     const uint32_t sq = (uint32_t)(slot - rowid * spr);
