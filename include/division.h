@@ -101,7 +101,9 @@ typedef struct div_plan {
                                7: small planes of any width (tile side 4, 8 or 16 after padding, at most 32 lanes per
                                   plane row, Q in {2,4,8}) in one launch: a CTA owns a run of planes of one sample,
                                   joins the sample's other CTAs through an arrival count and quantises the same
-                                  planes (second read from L1 / L2); taken when all its CTAs can be resident;
+                                  planes (second read from L1 / L2); taken when all its CTAs can be resident; also the
+                                  first choice for maps of such planes with W%4==0 below 56 MiB (bfloat16: below
+                                  32 MiB), as long as the flags exclude none of the kernels 2, 3, 6;
                                4: the same in two launches;
                                1: one launch, shared-memory ring, general kernel;  0: two-pass general kernels;
                                8: 1-D maps (h == 1; the appendix on 1D and 3D activation maps), W%4==0, B a power of two

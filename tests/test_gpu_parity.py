@@ -131,8 +131,8 @@ def small_input(n, c, h, w, x_dtype, seed):
 
 
 @pytest.mark.parametrize("case", SMALL, ids=lambda c: "x".join(map(str, c)))
-@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS],
-                         ids=["default", "lagged", "staged", "planes", "planes_pair", "general_ring", "two_pass"])
+@pytest.mark.parametrize("flags", [0, RING, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS],
+                         ids=["default", "strip_ring", "lagged", "staged", "planes", "planes_pair", "general_ring", "two_pass"])
 def test_small_cases_match_the_checker(case, flags):
     n, c, h, w, block, q, xd, ld = case
     x = small_input(n, c, h, w, xd, seed=n + c + h + w + block + q)
@@ -159,7 +159,8 @@ def test_fused_path_is_taken_where_expected():
         n, c, h, w, block, q, xd, ld = case
         strip_shape = w % 4 == 0 and min(block, max(h, w)) in (4, 8) and q in (2, 4, 8)
         if strip_shape:
-            assert fused[case] == 2 and lagged[case] == 3, case
+            # narrow planes (W <= 32 for B = 8) take the fused small-plane kernel by default, wider ones a strip kernel
+            assert fused[case] == (7 if planes_shape(case) else 2) and lagged[case] == 3, case
             # bulk copies need every sample, plane and band to start on a 16-byte boundary
             sx = 4 if xd == "f32" else 2
             b = min(block, max(h, w))
@@ -171,9 +172,10 @@ def test_fused_path_is_taken_where_expected():
         else:
             assert fused[case] in (0, 1) and lagged[case] == fused[case] and staged[case] == fused[case], case
         assert special[case] == (7 if planes_shape(case) else binding.div_plan_query(binding.make_desc(*case), NO_STRIP).fused), case
-    assert sum(1 for c in SMALL if fused[c] == 2) >= 12
+    assert sum(1 for c in SMALL if fused[c] == 2) >= 2
+    assert sum(1 for c in SMALL if binding.div_plan_query(binding.make_desc(*c), RING).fused == 2) >= 12
     assert sum(1 for c in SMALL if staged[c] == 6) >= 12
-    assert sum(1 for c in SMALL if fused[c] == 7) >= 5
+    assert sum(1 for c in SMALL if fused[c] == 7) >= 15
     assert sum(1 for c in SMALL if special[c] == 7) >= 12
     assert fused[(2, 4, 32, 32, 8, 1, "f32", "f32")] == 1          # Q = 1: general ring kernel
     assert fused[(2, 8, 14, 14, 8, 2, "f32", "f32")] == 7
@@ -186,6 +188,9 @@ def test_fused_path_is_taken_where_expected():
         d = binding.make_desc(*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype)
         nbytes = spec.numel * (4 if spec.x_dtype == "f32" else 2)
         first = 6 if (nbytes >= 56 * 2 ** 20 and spec.block == 8) else (3 if nbytes >= 20 * 2 ** 20 else 2)
+        narrow = planes_shape((*spec.shape, spec.block, spec.qbits, spec.x_dtype, spec.lfc_dtype))
+        if narrow and nbytes < 56 * 2 ** 20 and not (spec.x_dtype == "bf16" and nbytes >= 32 * 2 ** 20):
+            first = 7
         assert binding.div_plan_query(d).fused == (first if spec.w % 4 == 0 else 7), spec.label()
         assert binding.div_plan_query(d, LAGGED).fused == (3 if spec.w % 4 == 0 else 7), spec.label()
         assert binding.div_plan_query(d, RING).fused == (2 if spec.w % 4 == 0 else 7), spec.label()
@@ -208,7 +213,7 @@ def test_decompress_reads_a_checker_blob():
 def test_degenerate_inputs():
     # constant tensor: residual identically zero, Delta = 0, exact reconstruction
     x = np.full((2, 4, 16, 16), 1.7, dtype=np.float32)
-    for flags in (0, LAGGED, STAGED, TWO_PASS):
+    for flags in (0, RING, LAGGED, STAGED, TWO_PASS):
         codec, blob, xhat = run_gpu(x, 8, 2, 3, flags=flags)
         lfc, words, stats = split_blob(blob, codec.layout, "f32")
         assert not words.any() and not stats.any()
@@ -241,7 +246,7 @@ def test_same_seed_same_bytes_other_seed_other_codes():
     assert (wa != wc).mean() > 0.5
 
 
-@pytest.mark.parametrize("flags", [0, LAGGED, STAGED, NO_SPECIAL], ids=["strip_ring", "lagged", "staged", "planes_fused"])
+@pytest.mark.parametrize("flags", [RING, LAGGED, STAGED, NO_SPECIAL], ids=["strip_ring", "lagged", "staged", "planes_fused"])
 def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
     """Failure detection without a fault: the kernel waits for arrivals that never come, its 2 ms limit
     runs out, it records the timeout in the status word and returns; the context stays usable."""
@@ -251,7 +256,7 @@ def test_a_wait_that_cannot_end_gives_up_and_reports_it(flags):
         spec = synth.TensorSpec(0, 0, 8, 64, 14, 14, "relu", "f32", "f32", 8, 2)      # a small-plane map
     x = to_device(synth.make_input(spec), "f32")
     codec = binding.Codec(*spec.shape, spec.block, spec.qbits)
-    assert codec.plan(flags).fused == {0: 2, LAGGED: 3, STAGED: 6, NO_SPECIAL: 7}[flags]
+    assert codec.plan(flags).fused == {RING: 2, LAGGED: 3, STAGED: 6, NO_SPECIAL: 7}[flags]
     st = binding.lib().div_debug_compress_starved(
         ctypes.byref(codec.desc), ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(codec.blob.data_ptr()), codec.blob.numel(),
         ctypes.c_void_p(codec.workspace.data_ptr()), codec.workspace.numel(), 0, ctypes.c_void_p(binding.current_stream_handle()),
@@ -273,7 +278,7 @@ def test_guard_bands_stay_untouched():
     for case in [(2, 8, 14, 14, 8, 2, "f32", "f32"), (3, 4, 32, 32, 8, 2, "f32", "f32"), (3, 5, 7, 9, 4, 1, "f32", "f32"),
                  (2, 8, 32, 32, 8, 2, "bf16", "bf16")]:
         n, c, h, w, block, q, xd, ld = case
-        for flags in (0, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS):
+        for flags in (0, RING, LAGGED, STAGED, NO_SPECIAL, PLANES_PAIR, NO_STRIP, TWO_PASS):
             x = small_input(n, c, h, w, xd, seed=7)
             codec = binding.Codec(n, c, h, w, block, q, xd, ld)
             pad = 4096
@@ -326,7 +331,7 @@ def assert_sampled_parity(spec, seed, sample_ids, flags=0):
 def test_config0_full():
     spec = synth.config0()[0]
     x = synth.make_input(spec)
-    for flags in (0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
+    for flags in (0, RING, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
         assert_full_parity(x, spec.block, spec.qbits, 0, flags=flags)
 
 
@@ -369,7 +374,7 @@ def test_block_sum_order_on_every_path():
     x[0, 0, 0:8, 0:8] = tile
     x[1, 7, 8:16, 24:32] = tile
     x[2, 15, 24:32, 16:24] = tile.T
-    for flags in (0, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
+    for flags in (0, RING, LAGGED, STAGED, NO_SPECIAL, NO_STRIP, TWO_PASS):
         codec = assert_full_parity(x, 8, 2, seed=5, flags=flags)
         lfc, _, _ = split_blob(codec.blob.cpu().numpy(), codec.layout, "f32")
         assert lfc.reshape(3, 16, 4, 4)[0, 0, 0, 0] == np.float32(3.0 / 64.0)
