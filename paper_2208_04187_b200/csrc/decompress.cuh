@@ -65,6 +65,7 @@ struct DecFast {
     uint32_t H;
     uint32_t hwq, wq;    // quads per plane and per row
     uint32_t ipp;        // work items per plane = ceil(H/4) * (W/4)
+    uint32_t hq_count;   // ceil(H/4): SPREAD items take the rows hq, hq + hq_count, hq + 2 hq_count, hq + 3 hq_count
     uint32_t items;      // work items per sample = C * ipp
     FastDiv by_ipp;      // / ipp
     FastDiv by_wq;       // / (W/4)
@@ -144,7 +145,11 @@ __device__ __forceinline__ uint32_t quad_bits(const uint32_t* __restrict__ packe
     return (__ldg(reinterpret_cast<const uint8_t*>(packed) + (quad >> 1)) >> (4u * (uint32_t)(quad & 1u))) & 15u;
 }
 
-template <typename XT, typename LT, int Q, int QPT>
+// SPREAD: where a row is not a whole number of 32-byte sectors (28 fp32 columns: 112 bytes) the 4 rows of a work
+// item are taken hq_count rows apart instead of next to each other, so that the lanes of a warp write consecutive
+// rows with one store instruction (whole sectors) instead of pieces 4 rows apart; the rows of an item then lie in
+// different tiles, each with its own low-frequency value.
+template <typename XT, typename LT, int Q, int QPT, bool SPREAD>
 __global__ void __launch_bounds__(256)
 decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
@@ -159,20 +164,30 @@ decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
     const uint32_t rem = item - plane * d.ipp;
     const uint32_t hq = fdiv(rem, d.by_wq);
     const uint32_t wq = rem - hq * d.wq;
-    const uint32_t h0 = hq * 4u;
-    const float lf = Elem<LT>::load(lfc + ((size_t)n * d.C + plane) * d.TPP + (h0 >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
+    const uint32_t h0 = SPREAD ? hq : hq * 4u;
+    const uint32_t hstep = SPREAD ? d.hq_count : 1u;
+    const LT* lfc_p = lfc + ((size_t)n * d.C + plane) * d.TPP + ((wq * 4u) >> d.log2B);
     const uint64_t quad0 = (uint64_t)n * d.qps + plane * d.hwq + h0 * d.wq + wq;      // first row's quad
-    const uint32_t rows = min(4u, d.H - h0);
+    const uint32_t qstep = hstep * d.wq;
+    float lf[4];
     uint32_t bits[4];
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-        if ((uint32_t)r < rows) bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * d.wq);
+    for (int r = 0; r < 4; ++r) {
+        const uint32_t h = h0 + (uint32_t)r * hstep;
+        bits[r] = 0u;
+        lf[r] = 0.f;
+        if (h < d.H) {
+            bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * qstep);
+            if (SPREAD || r == 0) lf[r] = Elem<LT>::load(lfc_p + (h >> d.log2B) * d.Wb);
+        }
+        if (!SPREAD && r > 0) lf[r] = lf[0];              // 4 neighbouring rows from a multiple of 4 on share a tile
+    }
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-        if ((uint32_t)r < rows) {
+        if (h0 + (uint32_t)r * hstep < d.H) {
             const float4 hq4 = table.quad(bits[r]);
-            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * d.wq) * 4u, __fadd_rn(lf, hq4.x), __fadd_rn(lf, hq4.y),
-                            __fadd_rn(lf, hq4.z), __fadd_rn(lf, hq4.w));
+            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * qstep) * 4u, __fadd_rn(lf[r], hq4.x), __fadd_rn(lf[r], hq4.y),
+                            __fadd_rn(lf[r], hq4.z), __fadd_rn(lf[r], hq4.w));
         }
     }
 }

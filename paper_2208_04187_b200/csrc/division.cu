@@ -470,12 +470,17 @@ div_status div_decompress(const div_desc* desc, const void* comp_dev, size_t com
                 d.H = s.H;
                 d.hwq = s.HW / 4;
                 d.wq = s.W / 4;
-                d.ipp = ((s.H + 3u) / 4u) * d.wq;
+                d.hq_count = (s.H + 3u) / 4u;
+                d.ipp = d.hq_count * d.wq;
                 d.items = s.C * d.ipp;
                 d.by_ipp = make_fastdiv(d.ipp);
                 d.by_wq = make_fastdiv(d.wq);
                 dim3 grid((d.items + 255u) / 256u, s.N);
-                decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+                // rows that are not whole 32-byte sectors: the 4 rows of an item spread over the plane (see the kernel)
+                if ((s.W * (uint32_t)sizeof(XT)) % 32u != 0 && s.H >= 8u)
+                    decompress_quad_kernel<XT, LT, Q, DEC_QPT, true><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+                else
+                    decompress_quad_kernel<XT, LT, Q, DEC_QPT, false><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
             } else if (decompress_flat_ok(s)) {
                 DecFlat d;
                 d.qps = s.CHW / 4;
