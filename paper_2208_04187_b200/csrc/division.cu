@@ -683,12 +683,16 @@ div_status div_planegroup_decompress(const div_desc* desc, const void* comp_dev,
                 d.H = s.H;
                 d.hwq = s.HW / 4;
                 d.wq = s.W / 4;
-                d.ipp = ((s.H + 3u) / 4u) * d.wq;
+                d.hq_count = (s.H + 3u) / 4u;
+                d.ipp = d.hq_count * d.wq;
                 d.items = s.C * d.ipp;
                 d.by_ipp = make_fastdiv(d.ipp);
                 d.by_wq = make_fastdiv(d.wq);
                 dim3 grid((d.items + 255u) / 256u, s.N);
-                pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+                if ((s.W * (uint32_t)sizeof(XT)) % 32u != 0 && s.H >= 8u)
+                    pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT, true><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
+                else
+                    pg_decompress_quad_kernel<XT, LT, Q, DEC_QPT, false><<<grid, 256, 0, stream>>>(lfc, packed, stats, (XT*)xhat_dev, d);
             } else if (pg_decompress_flat_ok(s)) {
                 PgDecFlat d;
                 d.quads = s.total / 4;

@@ -502,7 +502,9 @@ __device__ __forceinline__ void pg_unpack_stats(uint32_t w, float& delta, float&
 
 // W % 4 == 0 and B a power of two >= 4: same tiling of the work as decompress_quad_kernel (a thread produces
 // the same 4 columns of 4 consecutive rows: one low-frequency value, one plane pair, one set of index arithmetic)
-template <typename XT, typename LT, int Q, int QPT>
+// SPREAD: as in decompress_quad_kernel (rows that are not whole 32-byte sectors: the 4 rows of an item lie
+// hq_count rows apart, each with its own tile's low-frequency value)
+template <typename XT, typename LT, int Q, int QPT, bool SPREAD>
 __global__ void __launch_bounds__(256)
 pg_decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                           const uint32_t* __restrict__ stats, XT* __restrict__ xhat, DecFast d) {
@@ -515,24 +517,34 @@ pg_decompress_quad_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict
     const uint32_t rem = item - plane * d.ipp;
     const uint32_t hq = fdiv(rem, d.by_wq);
     const uint32_t wq = rem - hq * d.wq;
-    const uint32_t h0 = hq * 4u;
+    const uint32_t h0 = SPREAD ? hq : hq * 4u;
+    const uint32_t hstep = SPREAD ? d.hq_count : 1u;
     const size_t gp = (size_t)n * d.C + plane;
-    const float lf = Elem<LT>::load(lfc + gp * d.TPP + (h0 >> d.log2B) * d.Wb + ((wq * 4u) >> d.log2B));
+    const LT* lfc_p = lfc + gp * d.TPP + ((wq * 4u) >> d.log2B);
     float delta, step;
     pg_unpack_stats(__ldg(stats + gp), delta, step);
     const uint64_t quad0 = (uint64_t)n * d.qps + plane * d.hwq + h0 * d.wq + wq;
-    const uint32_t rows = min(4u, d.H - h0);
+    const uint32_t qstep = hstep * d.wq;
     uint32_t bits[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-        if ((uint32_t)r < rows) bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * d.wq);
+    float lf[4];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
-        if ((uint32_t)r < rows) {
-            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * d.wq) * 4u, reconstruct(bits[r] & MASK, step, delta, lf),
-                            reconstruct((bits[r] >> Q) & MASK, step, delta, lf),
-                            reconstruct((bits[r] >> (2 * Q)) & MASK, step, delta, lf),
-                            reconstruct((bits[r] >> (3 * Q)) & MASK, step, delta, lf));
+        const uint32_t h = h0 + (uint32_t)r * hstep;
+        bits[r] = 0u;
+        lf[r] = 0.f;
+        if (h < d.H) {
+            bits[r] = quad_bits<Q>(packed, quad0 + (uint32_t)r * qstep);
+            if (SPREAD || r == 0) lf[r] = Elem<LT>::load(lfc_p + (h >> d.log2B) * d.Wb);
+        }
+        if (!SPREAD && r > 0) lf[r] = lf[0];
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        if (h0 + (uint32_t)r * hstep < d.H) {
+            Quad<XT>::store(xhat + (quad0 + (uint32_t)r * qstep) * 4u, reconstruct(bits[r] & MASK, step, delta, lf[r]),
+                            reconstruct((bits[r] >> Q) & MASK, step, delta, lf[r]),
+                            reconstruct((bits[r] >> (2 * Q)) & MASK, step, delta, lf[r]),
+                            reconstruct((bits[r] >> (3 * Q)) & MASK, step, delta, lf[r]));
         }
     }
 }
