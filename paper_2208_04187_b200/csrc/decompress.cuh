@@ -288,11 +288,20 @@ template <typename XT, typename LT, int Q, int QPT>
 __global__ void __launch_bounds__(256)
 decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ packed,
                        const float* __restrict__ stats, XT* __restrict__ xhat, DecFlat d) {
-    extern __shared__ uint32_t flat_smem[];
+    extern __shared__ __align__(16) uint32_t flat_smem[];
     uint2* quad_of = reinterpret_cast<uint2*>(flat_smem);            // quad inside a period -> where its 4 low-frequency values sit
     float* lfc_s = reinterpret_cast<float*>(flat_smem + d.table_words);   // low-frequency values of this CTA's planes
     __shared__ DeqTable<Q> table;
     const uint32_t n = blockIdx.y;
+    // the codes of this thread's quads are asked for first: their trip to memory overlaps the set-up below
+    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
+    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
+    uint32_t bits[QPT];
+#pragma unroll
+    for (int k = 0; k < QPT; ++k) {
+        const uint32_t q = q0 + k * 256u;
+        bits[k] = q < d.qps ? quad_bits<Q>(packed, sample_quad0 + q) : 0u;
+    }
     table.build(__ldg(stats + 2 * (size_t)n + 1), __ldg(stats + 2 * (size_t)n));
     for (uint32_t idx = threadIdx.x; idx < d.period; idx += 256u)
         quad_of[idx] = quad_table_entry(idx, d.HW, d.W, d.Wb, d.TPP, d.by_hw, d.by_w, d.by_b);
@@ -302,13 +311,11 @@ decompress_flat_kernel(const LT* __restrict__ lfc, const uint32_t* __restrict__ 
     const LT* lfc_n = lfc + ((size_t)n * d.C + plane0) * d.TPP;
     for (uint32_t idx = threadIdx.x; idx < nplanes * d.TPP; idx += 256u) lfc_s[idx] = Elem<LT>::load(lfc_n + idx);
     __syncthreads();
-    const uint64_t sample_quad0 = (uint64_t)n * d.qps;
-    const uint32_t q0 = blockIdx.x * (256u * QPT) + threadIdx.x;
 #pragma unroll
     for (int k = 0; k < QPT; ++k) {
         const uint32_t q = q0 + k * 256u;
         if (q < d.qps) {
-            const float4 hq = table.quad(quad_bits<Q>(packed, sample_quad0 + q));
+            const float4 hq = table.quad(bits[k]);
             const float hv[4] = {hq.x, hq.y, hq.z, hq.w};
             const uint32_t grp = fdiv(q, d.by_period);
             const uint2 ent = quad_of[q - grp * d.period];
