@@ -1,5 +1,5 @@
-// Compress kernels for maps with small planes whose width is not a multiple of 4 (the 14 x 14 and
-// 7 x 7 maps of the ImageNet networks): DIVISION Sec. 4.1; Algorithm 1, forward loop.
+// Compress kernels for maps of small planes of any width (the 14 x 14 and 7 x 7 maps of the ImageNet networks;
+// also the first choice for planes up to 32 wide below 56 MiB): DIVISION Sec. 4.1; Algorithm 1, forward loop.
 //
 // plane_fused_kernel does both halves in one launch (see there); where its CTAs cannot all be resident the pair
 // below runs instead.  Two launches, no dependency inside a kernel:
@@ -9,13 +9,15 @@
 // The second kernel reads x again; these maps are a few tens of MB, so the second read comes from the
 // 126 MB L2 (larger tensors are still handled correctly, at the price of reading x twice from HBM).
 //
-// plane_stats_kernel: a lane owns one tile column of one plane (P2 lanes per tile, tiles_per_row * P2
-// lanes per plane, several planes per warp): per band it loads its column's rows, sums them with the
-// balanced tree, meets the other columns of the tile with xor shuffles (the same tree across columns),
-// and keeps the extremes of its column.
-// plane_quant_kernel: one thread per 4 consecutive elements of the flat sample (they may lie in
-// different tiles, rows or planes): where their 4 low-frequency values sit comes from the quad table in shared
-// memory (one 8-byte entry per quad of a period of lcm(HW, 4) elements), the arithmetic of Eq. 9 runs on packed pairs.
+// First half (plane_half1, used by plane_stats_kernel and plane_fused_kernel): a lane owns two adjacent columns
+// of one tile of one plane (P2 / 2 lanes per tile, several planes per warp): per band it loads its columns' rows
+// (one 8-byte load per row where W and B are even, else two loads), sums each column with the balanced tree,
+// meets the other columns of the tile with xor shuffles (the same tree across columns), and keeps the extremes
+// of its columns.
+// Second half (plane_quant_kernel, plane_fused_kernel): one thread per 4 consecutive elements of the flat sample
+// (they may lie in different tiles, rows or planes): where their 4 low-frequency values sit comes from the quad
+// table in shared memory (one 8-byte entry per quad of a period of lcm(HW, 4) elements), the arithmetic of Eq. 9
+// runs on packed pairs.
 #pragma once
 
 #include "decompress.cuh"   // quad table, flat_planes_per_cta, flat_smem_bytes
