@@ -128,12 +128,14 @@ line_quant_kernel(const XT* __restrict__ x, const LT* __restrict__ lfc, const ui
 }
 
 // One launch for both halves.  CTA (b, n) owns the rows [b * rpc, (b + 1) * rpc) of sample n:
-//   1. block means, stored low-frequency values and residual extremes of its rows, exactly as line_stats_kernel;
+//   1. block means, stored low-frequency values and residual extremes of its rows: the same values as
+//      line_stats_kernel in another layout (a lane owns a segment of min(B, 16) consecutive elements of one block);
 //      the CTA's extremes are folded into the sample's slot (two reductions without an answer), then, behind a
 //      release fence, the CTA is counted as arrived;
 //   2. thread 0 waits (bounded) until all CTAs of the sample have arrived and derives (delta, Delta, scale);
-//   3. Eq. 9 and packing of the same rows as line_quant_kernel: x is read a second time (it is still in this
-//      SM's L1 or in the L2), the low-frequency values are the ones this CTA stored in step 1.
+//   3. Eq. 9 and packing of the same rows, segment by segment (one low-frequency load and one counter per segment):
+//      x is read a second time (it is still in this SM's L1 or in the L2), the low-frequency values are the ones
+//      this CTA stored in step 1.
 // The launch is cooperative so that the CTAs a wait depends on are resident; no grid-wide barrier is used.
 struct LineFused {
     uint32_t rpc;                 // rows per CTA

@@ -5,6 +5,9 @@
 //                        axis, then down the rows, then across the columns), stored low-frequency value,
 //                        residual extremes -> per-sample min / max keys in the scratch slots
 //   lfc_stats3d_warp_kernel  the same with a lane per block column (blocks of padded side <= 32): coalesced loads
+//   lfc_stats3d_strip_kernel, quant3d_strip_kernel, decompress3d_strip_kernel
+//                        W % 4 == 0 and B = 4 or 8: a lane per strip of 4 adjacent columns of one block (16-byte
+//                        accesses), the default for such shapes
 //   quant_pack3d_kernel  one thread per packed 32-bit word
 //   decompress3d_kernel  one thread per packed 32-bit word
 // x is read twice by compress (the second time from L2 when the tensor fits).
